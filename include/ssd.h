@@ -1,0 +1,180 @@
+/*
+ * libssd -- decision kernels of CTC-draft self-speculative decoding for LLM-based ASR.
+ *
+ * The library computes, on one CUDA device, what wraps the LLM forward pass in the method:
+ *   stage 1 (ssd_ctc_draft, ssd_entropy_gate): from the CTC head's logits, per-frame
+ *     log-sum-exp, entropy and greedy argmax; the collapsed draft hypothesis; the
+ *     utterance-level entropy gate;
+ *   stage 2 (ssd_verify): from the LLM's logits at the draft positions, each draft token's
+ *     log-likelihood, the relaxed acceptance rule and the accepted prefix length.
+ *
+ * Conventions for every call
+ *   - All array pointers are DEVICE pointers owned by the caller unless a comment says
+ *     "host".  The library allocates nothing, frees nothing and never synchronises: work is
+ *     enqueued on `stream` (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ *   - A batch is ragged: utterance b owns rows [off[b], off[b+1]) of a row-major matrix with
+ *     `ld` elements between consecutive rows (ld >= V).  off is int64, off[0] = 0,
+ *     off[B] = number of rows.  The row count is also passed as a host scalar so that no
+ *     device-to-host read is needed.  B = 0, empty utterances and zero rows are legal.
+ *   - Logits are SSD_F32 (IEEE binary32) or SSD_BF16 (bfloat16).  The matrix base must be
+ *     aligned to the element size.  All accumulation is fp32.  -inf is a legal (masked)
+ *     logit; NaN, +inf or a row of only -inf set SSD_UTT_NONFINITE for the utterance and
+ *     leave that row's float outputs unspecified.
+ *   - Return value: SSD_OK or an error found on the host before anything was enqueued
+ *     (nothing is written in that case).  Problems only visible in the data are reported
+ *     per utterance in `utt_status` (bit set, no trap, nothing out of bounds is touched).
+ *   - Ties of the argmax go to the lowest index.  Entropy is in nats.
+ */
+#ifndef SSD_H_
+#define SSD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { SSD_F32 = 0, SSD_BF16 = 1 } ssd_dtype;
+
+/* return codes */
+enum {
+    SSD_OK = 0,
+    SSD_ERR_NULL = 1,      /* a required pointer is NULL */
+    SSD_ERR_ARG = 2,       /* negative size, ld < V, blank_id outside [0,V), bad option ... */
+    SSD_ERR_DTYPE = 3,     /* dtype is neither SSD_F32 nor SSD_BF16 */
+    SSD_ERR_WORKSPACE = 4, /* workspace NULL or smaller than the *_workspace_bytes() answer */
+    SSD_ERR_CUDA = 5,      /* a CUDA runtime call failed; see ssd_last_cuda_error() */
+    SSD_ERR_ALIGN = 6      /* logits base not aligned to the element size */
+};
+
+/* bits of utt_status[b] */
+enum {
+    SSD_UTT_NONFINITE = 1u,     /* a row of the utterance held NaN / +inf or only -inf */
+    SSD_UTT_BAD_DRAFT_ID = 2u,  /* a draft id outside [0,V): treated as rejected, never read */
+    SSD_UTT_BAD_OFFSETS = 4u,   /* off[b] < 0, off[b+1] < off[b] or off[b+1] > rows: utterance
+                                   treated as empty and never accepted */
+    SSD_UTT_INTERNAL = 0x80000000u /* a bounded wait inside a kernel ran out while this utterance
+                                      was processed: discard every output of the call */
+};
+
+/*
+ * Optional launch controls, for tuning and measurement.  Pass NULL for the defaults.  Zero in
+ * a field means "choose automatically".  The struct is read on the host during the call only.
+ */
+typedef struct ssd_launch_opts {
+    int32_t kernel;       /* 0 auto; 1 plain-load kernels; 2 bulk-copy (TMA) pipelined kernels */
+    int32_t ctas;         /* grid size of the streaming kernel */
+    int32_t warps;        /* compute warps per CTA of the streaming kernel */
+    int32_t stages;       /* shared-memory pipeline depth */
+    int32_t stage_bytes;  /* bytes per pipeline stage (verify) / rows per stage (ctc_draft) */
+    int32_t split;        /* verify: column spans per logits row */
+    void *ev_begin;       /* cudaEvent_t recorded just before the streaming kernel, or NULL */
+    void *ev_end;         /* cudaEvent_t recorded just after the streaming kernel, or NULL */
+} ssd_launch_opts;
+
+/* Human-readable name of a return code (static storage). */
+const char *ssd_status_string(int32_t status);
+
+/* cudaError_t of the last failing CUDA call seen by this thread (0 if none). */
+int32_t ssd_last_cuda_error(void);
+
+/* Library version, major*10000 + minor*100 + patch. */
+int32_t ssd_version(void);
+
+/* Bytes of device scratch the calls below need for these sizes and options (may be 0). */
+size_t ssd_ctc_draft_workspace_bytes(int32_t B, int64_t N, int32_t V, ssd_dtype dtype,
+                                     const ssd_launch_opts *opts);
+size_t ssd_verify_workspace_bytes(int32_t B, int64_t M, int32_t V, ssd_dtype dtype,
+                                  const ssd_launch_opts *opts);
+
+/*
+ * Stage 1: CTC draft.  Section 2.1 of the paper.
+ *
+ * For every frame t (row of `logits`, V = size of the augmented vocabulary incl. blank):
+ *   frame_lse[t]     = log sum_a exp(x_ta)          (so log p(a|h_t) = x_ta - frame_lse[t])
+ *   frame_entropy[t] = sum_a -p(a|h_t) log p(a|h_t)                     (Eq. 3, left side)
+ *   frame_argmax[t]  = argmax_a p(a|h_t)                                (Eq. 2)
+ * and for every utterance b the draft hypothesis B(argmax path): consecutive duplicates
+ * merged, then blanks removed (in this order, the mapping B of Section 2.1):
+ *   draft_tokens[frame_off[b] + k], k < draft_len[b]   the first draft_len[b] tokens
+ *   draft_frames[frame_off[b] + k]                     frame index (within the utterance) that
+ *                                                      emitted token k            (nullable)
+ *   draft_full_len[b] = U, the uncapped length; draft_len[b] = min(U, max_draft_len)
+ *   utt_max_entropy[b] = max_t frame_entropy[t] over the utterance (0 if it has no frames)
+ *
+ * logits         [N, ld] dtype, read once.                          frame_off [B+1] int64
+ * frame_entropy  [N] f32   frame_argmax [N] i32   frame_lse [N] f32 (nullable)
+ * frame_logprob  [N, ld] f32 dense log-softmax x - lse (nullable; for inspection and tests:
+ *                it writes 4*N*V bytes and is not part of the timed path)
+ * draft_tokens   [N] i32 (U <= T guarantees the capacity; entries past draft_len[b] inside an
+ *                utterance's range are left untouched)
+ * draft_len, draft_full_len [B] i32   utt_max_entropy [B] f32   utt_status [B] u32 (overwritten)
+ * workspace      at least ssd_ctc_draft_workspace_bytes(...) bytes, 256-byte aligned; may be
+ *                NULL when that is 0.
+ * Errors: SSD_ERR_NULL, SSD_ERR_ARG (B,N < 0; V < 1; ld < V; blank_id outside [0,V);
+ * max_draft_len < 0), SSD_ERR_DTYPE, SSD_ERR_ALIGN, SSD_ERR_WORKSPACE, SSD_ERR_CUDA.
+ */
+int32_t ssd_ctc_draft(const void *logits, ssd_dtype dtype, int32_t V, int64_t ld,
+                      const int64_t *frame_off, int32_t B, int64_t N,
+                      int32_t blank_id, int32_t max_draft_len,
+                      float *frame_entropy, int32_t *frame_argmax, float *frame_lse,
+                      float *frame_logprob,
+                      int32_t *draft_tokens, int32_t *draft_frames,
+                      int32_t *draft_len, int32_t *draft_full_len,
+                      float *utt_max_entropy, uint32_t *utt_status,
+                      void *workspace, size_t workspace_bytes, void *stream,
+                      const ssd_launch_opts *opts);
+
+/*
+ * Stage 1 decision: the entropy gate.  Eq. 3 of the paper: the draft of utterance b is
+ * accepted as final iff frame_entropy[t] < tau_ctc for ALL of its frames (strict).
+ *   gate_accept[b]  = 1 / 0          (an utterance without frames passes iff 0 < tau_ctc;
+ *                                     a NaN entropy or malformed offsets never pass)
+ *   max_entropy[b]  = max over the utterance's frames (0 if none)
+ *   argmax_frame[b] = first frame attaining it, -1 if none                     (nullable)
+ * frame_entropy [N] f32 may come from ssd_ctc_draft or anywhere else.
+ * Errors: SSD_ERR_NULL, SSD_ERR_ARG, SSD_ERR_CUDA.
+ */
+int32_t ssd_entropy_gate(const float *frame_entropy, const int64_t *frame_off,
+                         int32_t B, int64_t N, float tau_ctc,
+                         uint8_t *gate_accept, float *max_entropy, int32_t *argmax_frame,
+                         void *stream);
+
+/*
+ * Stage 2: LLM verification of the draft.  Eq. 5 and Section 2.3 of the paper.
+ *
+ * Row i of `logits` (V = LLM vocabulary) is the LLM's output distribution that predicts
+ * draft token i of its utterance (the caller has already aligned positions, and passes only
+ * the rows at draft positions).  For every row:
+ *   row_lse[i]    = log sum_v exp(x_iv)                                        (nullable)
+ *   token_logp[i] = x[i, draft_ids[i]] - row_lse[i]   = log p(y_i | y_<i, g)   (Eq. 5)
+ * Position i is rejected iff p <= tau_slm, evaluated as token_logp[i] <= log(tau_slm)
+ * (accepted iff p > tau_slm, Eq. 5).  For every utterance b with K_b rows:
+ *   accepted_len[b] = index (0-based, within the utterance) of the first rejected position,
+ *                     K_b if none: the verified prefix has accepted_len[b] tokens and AR
+ *                     decoding would resume at that position (the paper's j is this + 1)
+ *   all_accepted[b] = (accepted_len[b] == K_b): Eq. 5 holds (vacuously for K_b = 0)
+ * tau_slm <= 0 rejects nothing; tau_slm >= 1 rejects everything.  A NaN likelihood or a
+ * draft id outside [0,V) is a rejected position.
+ * skip [B] u8 (nullable): nonzero = the utterance was already accepted by the gate; its rows
+ * are not read, accepted_len = K_b, all_accepted = 1, its token_logp / row_lse untouched.
+ *
+ * logits [M, ld] dtype, read once    tok_off [B+1] int64    draft_ids [M] i32
+ * token_logp [M] f32   accepted_len [B] i32   all_accepted [B] u8   utt_status [B] u32
+ * workspace: at least ssd_verify_workspace_bytes(...) bytes, 256-byte aligned.
+ * Errors: SSD_ERR_NULL, SSD_ERR_ARG, SSD_ERR_DTYPE, SSD_ERR_ALIGN, SSD_ERR_WORKSPACE,
+ * SSD_ERR_CUDA.
+ */
+int32_t ssd_verify(const void *logits, ssd_dtype dtype, int32_t V, int64_t ld,
+                   const int64_t *tok_off, const int32_t *draft_ids, int32_t B, int64_t M,
+                   float tau_slm, const uint8_t *skip,
+                   float *token_logp, float *row_lse,
+                   int32_t *accepted_len, uint8_t *all_accepted, uint32_t *utt_status,
+                   void *workspace, size_t workspace_bytes, void *stream,
+                   const ssd_launch_opts *opts);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SSD_H_ */

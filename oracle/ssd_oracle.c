@@ -211,7 +211,7 @@ int32_t ssd_ref_entropy_gate(const double *frame_entropy, const int64_t *frame_o
  * Stage 2 on a ragged batch: rows [tok_off[b], tok_off[b+1]) of the [M, ld] LLM logits
  * are the distributions that predict draft tokens 0..K_b-1 of utterance b.
  *   token_logp[i] = x[i, draft_ids[i]] - lse_i                         (Eq. 5, in log)
- *   reject_i      = p_i <= tau_slm  (p_i = exp(token_logp[i]))         (Section 2.3)
+ *   reject_i      = not (p_i > tau_slm), i.e. p_i <= tau_slm, or p_i is NaN  (Eq. 5; 2.3)
  *   accepted_len  = first rejected position (0-based), K_b if none
  *   all_accepted  = (accepted_len == K_b)                              (Eq. 5 holds)
  * The decision is also evaluated as token_logp <= log(tau); a disagreement sets
@@ -262,8 +262,10 @@ int32_t ssd_ref_verify(const void *logits, int32_t dtype, int32_t V, int64_t ld,
                 double lp = ref_load(logits, dtype, r * ld + id) - l;
                 double p = exp(lp);
                 token_logp[r] = lp;
-                reject = (p <= tau_slm);
-                int reject_log = (lp <= log_tau);
+                /* Eq. 5 accepts iff p > tau; "not accepted" also covers a NaN likelihood,
+                 * for which p <= tau (Section 2.3) would be false as well */
+                reject = !(p > tau_slm);
+                int reject_log = !(lp > log_tau);
                 if (tau_slm <= 0.0) { reject = 0; reject_log = 0; }
                 if (reject != reject_log) st |= SSD_REF_UTT_LOGP_P_DISAGREE;
             }

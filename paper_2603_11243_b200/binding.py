@@ -1,0 +1,203 @@
+"""Thin Python binding of libssd's C ABI (argument marshalling only).
+
+Every function here takes torch tensors that already live on the CUDA device, passes their
+addresses to the C entry point of the same name and returns the output tensors; all
+computation happens in the library's CUDA kernels.  There is no CPU fallback: importing this
+module without a built libssd.so, or calling it with host tensors, raises.
+"""
+import ctypes as C
+import os
+from typing import Dict, Optional
+
+import torch
+
+F32, BF16 = 0, 1
+UTT_NONFINITE, UTT_BAD_DRAFT_ID, UTT_BAD_OFFSETS, UTT_INTERNAL = 1, 2, 4, 0x80000000
+OK, ERR_NULL, ERR_ARG, ERR_DTYPE, ERR_WORKSPACE, ERR_CUDA, ERR_ALIGN = range(7)
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libssd.so")
+
+
+class SsdError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = lib().ssd_status_string(code).decode()
+        if code == ERR_CUDA:
+            msg += " (cudaError %d)" % lib().ssd_last_cuda_error()
+        super().__init__("%s: %s" % (where, msg))
+
+
+class LaunchOpts(C.Structure):
+    """Mirror of ssd_launch_opts (include/ssd.h)."""
+    _fields_ = [("kernel", C.c_int32), ("ctas", C.c_int32), ("warps", C.c_int32),
+                ("stages", C.c_int32), ("stage_bytes", C.c_int32), ("split", C.c_int32),
+                ("ev_begin", C.c_void_p), ("ev_end", C.c_void_p)]
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(
+                "libssd.so is not built: run `python -m paper_2603_11243_b200.build` "
+                "(needs nvcc); there is no fallback path")
+        L = C.CDLL(LIB_PATH)
+        L.ssd_status_string.restype = C.c_char_p
+        L.ssd_status_string.argtypes = [C.c_int32]
+        L.ssd_last_cuda_error.restype = C.c_int32
+        L.ssd_version.restype = C.c_int32
+        for f in (L.ssd_ctc_draft_workspace_bytes, L.ssd_verify_workspace_bytes):
+            f.restype = C.c_size_t
+            f.argtypes = [C.c_int32, C.c_int64, C.c_int32, C.c_int, C.c_void_p]
+        vp, i32, i64 = C.c_void_p, C.c_int32, C.c_int64
+        L.ssd_ctc_draft.restype = i32
+        L.ssd_ctc_draft.argtypes = [vp, C.c_int, i32, i64, vp, i32, i64, i32, i32,
+                                    vp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
+                                    vp, C.c_size_t, vp, vp]
+        L.ssd_entropy_gate.restype = i32
+        L.ssd_entropy_gate.argtypes = [vp, vp, i32, i64, C.c_float, vp, vp, vp, vp]
+        L.ssd_verify.restype = i32
+        L.ssd_verify.argtypes = [vp, C.c_int, i32, i64, vp, vp, i32, i64, C.c_float, vp,
+                                 vp, vp, vp, vp, vp, vp, C.c_size_t, vp, vp]
+        _lib = L
+    return _lib
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError("logits must be float32 or bfloat16, got %s" % t.dtype)
+
+
+def _dev(t: Optional[torch.Tensor], name: str):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("%s must be a CUDA tensor: libssd has no host path" % name)
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _opts(o: Optional[LaunchOpts]):
+    return None if o is None else C.cast(C.pointer(o), C.c_void_p)
+
+
+def _rows_ld(logits: torch.Tensor):
+    if logits.dim() != 2 or logits.stride(1) != 1:
+        raise ValueError("logits must be a 2-D row-major matrix (unit stride along the vocabulary)")
+    return logits.shape[0], (logits.stride(0) if logits.shape[0] > 1 else max(logits.stride(0), logits.shape[1]))
+
+
+def ssd_ctc_draft_workspace_bytes(B, N, V, dtype_code, opts=None) -> int:
+    return int(lib().ssd_ctc_draft_workspace_bytes(B, N, V, dtype_code, _opts(opts)))
+
+
+def ssd_verify_workspace_bytes(B, M, V, dtype_code, opts=None) -> int:
+    return int(lib().ssd_verify_workspace_bytes(B, M, V, dtype_code, _opts(opts)))
+
+
+def alloc_ctc_outputs(N: int, B: int, device, logprob_ld: int = 0) -> Dict[str, torch.Tensor]:
+    e = lambda n, dt: torch.empty((n,), dtype=dt, device=device)
+    out = dict(frame_entropy=e(N, torch.float32), frame_argmax=e(N, torch.int32),
+               frame_lse=e(N, torch.float32), draft_tokens=e(N, torch.int32),
+               draft_frames=e(N, torch.int32), draft_len=e(B, torch.int32),
+               draft_full_len=e(B, torch.int32), utt_max_entropy=e(B, torch.float32),
+               utt_status=e(B, torch.int32))
+    if logprob_ld:
+        out["frame_logprob"] = torch.empty((N, logprob_ld), dtype=torch.float32, device=device)
+    return out
+
+
+def ssd_ctc_draft(logits: torch.Tensor, frame_off: torch.Tensor, blank_id: int,
+                  max_draft_len: int, V: Optional[int] = None, out=None, want_logprob=False,
+                  opts: Optional[LaunchOpts] = None) -> Dict[str, torch.Tensor]:
+    """Stage 1 (Section 2.1, Eq. 2, Eq. 3): frame statistics and the collapsed draft."""
+    N, ld = _rows_ld(logits)
+    V = logits.shape[1] if V is None else V
+    B = frame_off.shape[0] - 1
+    if frame_off.dtype != torch.int64:
+        raise TypeError("frame_off must be int64")
+    if out is None:
+        out = alloc_ctc_outputs(N, B, logits.device, ld if want_logprob else 0)
+    rc = lib().ssd_ctc_draft(
+        _dev(logits, "logits"), _dtype_code(logits), V, ld, _dev(frame_off, "frame_off"), B, N,
+        blank_id, max_draft_len, _dev(out["frame_entropy"], "frame_entropy"),
+        _dev(out["frame_argmax"], "frame_argmax"), _dev(out.get("frame_lse"), "frame_lse"),
+        _dev(out.get("frame_logprob"), "frame_logprob"),
+        _dev(out["draft_tokens"], "draft_tokens"), _dev(out.get("draft_frames"), "draft_frames"),
+        _dev(out["draft_len"], "draft_len"), _dev(out["draft_full_len"], "draft_full_len"),
+        _dev(out["utt_max_entropy"], "utt_max_entropy"), _dev(out["utt_status"], "utt_status"),
+        None, 0, _stream(), _opts(opts))
+    if rc != OK:
+        raise SsdError(rc, "ssd_ctc_draft")
+    return out
+
+
+def alloc_gate_outputs(B: int, device) -> Dict[str, torch.Tensor]:
+    return dict(gate_accept=torch.empty((B,), dtype=torch.uint8, device=device),
+                max_entropy=torch.empty((B,), dtype=torch.float32, device=device),
+                argmax_frame=torch.empty((B,), dtype=torch.int32, device=device))
+
+
+def ssd_entropy_gate(frame_entropy: torch.Tensor, frame_off: torch.Tensor, tau_ctc: float,
+                     out=None) -> Dict[str, torch.Tensor]:
+    """The entropy gate (Eq. 3): accept iff every frame entropy is below tau_ctc."""
+    B, N = frame_off.shape[0] - 1, frame_entropy.shape[0]
+    if frame_entropy.dtype != torch.float32 or frame_off.dtype != torch.int64:
+        raise TypeError("frame_entropy must be float32 and frame_off int64")
+    if out is None:
+        out = alloc_gate_outputs(B, frame_entropy.device)
+    rc = lib().ssd_entropy_gate(
+        _dev(frame_entropy, "frame_entropy"), _dev(frame_off, "frame_off"), B, N,
+        C.c_float(tau_ctc), _dev(out["gate_accept"], "gate_accept"),
+        _dev(out["max_entropy"], "max_entropy"), _dev(out.get("argmax_frame"), "argmax_frame"),
+        _stream())
+    if rc != OK:
+        raise SsdError(rc, "ssd_entropy_gate")
+    return out
+
+
+def alloc_verify_outputs(M: int, B: int, device, workspace_bytes: int) -> Dict[str, torch.Tensor]:
+    e = lambda n, dt: torch.empty((n,), dtype=dt, device=device)
+    return dict(token_logp=e(M, torch.float32), row_lse=e(M, torch.float32),
+                accepted_len=e(B, torch.int32), all_accepted=e(B, torch.uint8),
+                utt_status=e(B, torch.int32),
+                workspace=torch.empty((max(workspace_bytes, 256),), dtype=torch.uint8,
+                                      device=device))
+
+
+def ssd_verify(logits: torch.Tensor, tok_off: torch.Tensor, draft_ids: torch.Tensor,
+               tau_slm: float, skip: Optional[torch.Tensor] = None, V: Optional[int] = None,
+               out=None, opts: Optional[LaunchOpts] = None) -> Dict[str, torch.Tensor]:
+    """Stage 2 (Eq. 5, Section 2.3): draft-token log-likelihoods and the accepted prefix."""
+    M, ld = _rows_ld(logits)
+    V = logits.shape[1] if V is None else V
+    B = tok_off.shape[0] - 1
+    if tok_off.dtype != torch.int64 or draft_ids.dtype != torch.int32:
+        raise TypeError("tok_off must be int64 and draft_ids int32")
+    if skip is not None and skip.dtype != torch.uint8:
+        raise TypeError("skip must be uint8")
+    code = _dtype_code(logits)
+    if out is None:
+        out = alloc_verify_outputs(M, B, logits.device,
+                                   ssd_verify_workspace_bytes(B, M, V, code, opts))
+    ws = out["workspace"]
+    rc = lib().ssd_verify(
+        _dev(logits, "logits"), code, V, ld, _dev(tok_off, "tok_off"),
+        _dev(draft_ids, "draft_ids"), B, M, C.c_float(tau_slm), _dev(skip, "skip"),
+        _dev(out["token_logp"], "token_logp"), _dev(out.get("row_lse"), "row_lse"),
+        _dev(out["accepted_len"], "accepted_len"), _dev(out["all_accepted"], "all_accepted"),
+        _dev(out["utt_status"], "utt_status"), _dev(ws, "workspace"), ws.numel(), _stream(),
+        _opts(opts))
+    if rc != OK:
+        raise SsdError(rc, "ssd_verify")
+    return out

@@ -1,0 +1,111 @@
+// The C ABI of libssd: argument validation and dispatch.  Every step of the path runs in the
+// kernels of ssd_ctc.cu and ssd_verify.cu; nothing here computes.
+#include "ssd_common.cuh"
+
+namespace ssd {
+static thread_local int32_t t_last_cuda_error = 0;
+void record_cuda_error(cudaError_t e) { t_last_cuda_error = (int32_t)e; }
+}  // namespace ssd
+
+using namespace ssd;
+
+extern "C" {
+
+const char *ssd_status_string(int32_t status) {
+    switch (status) {
+        case SSD_OK: return "SSD_OK";
+        case SSD_ERR_NULL: return "SSD_ERR_NULL: a required pointer is NULL";
+        case SSD_ERR_ARG: return "SSD_ERR_ARG: invalid size, leading dimension, id or option";
+        case SSD_ERR_DTYPE: return "SSD_ERR_DTYPE: dtype must be SSD_F32 or SSD_BF16";
+        case SSD_ERR_WORKSPACE: return "SSD_ERR_WORKSPACE: workspace missing, misaligned or too small";
+        case SSD_ERR_CUDA: return "SSD_ERR_CUDA: a CUDA runtime call failed";
+        case SSD_ERR_ALIGN: return "SSD_ERR_ALIGN: logits not aligned to the element size";
+        default: return "unknown status";
+    }
+}
+
+int32_t ssd_last_cuda_error(void) { return t_last_cuda_error; }
+
+int32_t ssd_version(void) { return 100; }
+
+size_t ssd_ctc_draft_workspace_bytes(int32_t B, int64_t N, int32_t V, ssd_dtype dtype,
+                                     const ssd_launch_opts *opts) {
+    (void)B; (void)N; (void)V; (void)dtype; (void)opts;
+    return 0;
+}
+
+size_t ssd_verify_workspace_bytes(int32_t B, int64_t M, int32_t V, ssd_dtype dtype,
+                                  const ssd_launch_opts *opts) {
+    if (B < 0 || M < 0 || V < 1 || (dtype != SSD_F32 && dtype != SSD_BF16)) return 0;
+    VerifyPlan plan;
+    if (plan_verify(B, M, V, dtype, opts, &plan) != SSD_OK) return 0;
+    return plan.workspace_bytes;
+}
+
+int32_t ssd_ctc_draft(const void *logits, ssd_dtype dtype, int32_t V, int64_t ld,
+                      const int64_t *frame_off, int32_t B, int64_t N,
+                      int32_t blank_id, int32_t max_draft_len,
+                      float *frame_entropy, int32_t *frame_argmax, float *frame_lse,
+                      float *frame_logprob,
+                      int32_t *draft_tokens, int32_t *draft_frames,
+                      int32_t *draft_len, int32_t *draft_full_len,
+                      float *utt_max_entropy, uint32_t *utt_status,
+                      void *workspace, size_t workspace_bytes, void *stream,
+                      const ssd_launch_opts *opts) {
+    (void)workspace; (void)workspace_bytes;
+    if (dtype != SSD_F32 && dtype != SSD_BF16) return SSD_ERR_DTYPE;
+    if (B < 0 || N < 0 || V < 1 || ld < V || blank_id < 0 || blank_id >= V || max_draft_len < 0)
+        return SSD_ERR_ARG;
+    if (!frame_off) return SSD_ERR_NULL;
+    if (N > 0 && (!logits || !frame_entropy || !frame_argmax || !draft_tokens)) return SSD_ERR_NULL;
+    if (B > 0 && (!draft_len || !draft_full_len || !utt_max_entropy || !utt_status))
+        return SSD_ERR_NULL;
+    const int es = dtype == SSD_F32 ? 4 : 2;
+    if (reinterpret_cast<uintptr_t>(logits) % es) return SSD_ERR_ALIGN;
+    Launch L{static_cast<cudaStream_t>(stream), opts};
+    int rc = launch_ctc_rows(logits, dtype, V, ld, N, frame_off, B, frame_entropy, frame_argmax,
+                             frame_lse, frame_logprob, utt_status, L);
+    if (rc != SSD_OK) return rc;
+    return launch_collapse(frame_argmax, frame_entropy, frame_off, B, N, blank_id, max_draft_len,
+                           draft_tokens, draft_frames, draft_len, draft_full_len,
+                           utt_max_entropy, utt_status, L.stream);
+}
+
+int32_t ssd_entropy_gate(const float *frame_entropy, const int64_t *frame_off,
+                         int32_t B, int64_t N, float tau_ctc,
+                         uint8_t *gate_accept, float *max_entropy, int32_t *argmax_frame,
+                         void *stream) {
+    if (B < 0 || N < 0) return SSD_ERR_ARG;
+    if (!frame_off) return SSD_ERR_NULL;
+    if (N > 0 && !frame_entropy) return SSD_ERR_NULL;
+    if (B > 0 && (!gate_accept || !max_entropy)) return SSD_ERR_NULL;
+    return launch_gate(frame_entropy, frame_off, B, N, tau_ctc, gate_accept, max_entropy,
+                       argmax_frame, static_cast<cudaStream_t>(stream));
+}
+
+int32_t ssd_verify(const void *logits, ssd_dtype dtype, int32_t V, int64_t ld,
+                   const int64_t *tok_off, const int32_t *draft_ids, int32_t B, int64_t M,
+                   float tau_slm, const uint8_t *skip,
+                   float *token_logp, float *row_lse,
+                   int32_t *accepted_len, uint8_t *all_accepted, uint32_t *utt_status,
+                   void *workspace, size_t workspace_bytes, void *stream,
+                   const ssd_launch_opts *opts) {
+    if (dtype != SSD_F32 && dtype != SSD_BF16) return SSD_ERR_DTYPE;
+    if (B < 0 || M < 0 || V < 1 || ld < V) return SSD_ERR_ARG;
+    if (!tok_off) return SSD_ERR_NULL;
+    if (M > 0 && (!logits || !draft_ids || !token_logp)) return SSD_ERR_NULL;
+    if (B > 0 && (!accepted_len || !all_accepted || !utt_status)) return SSD_ERR_NULL;
+    const int es = dtype == SSD_F32 ? 4 : 2;
+    if (reinterpret_cast<uintptr_t>(logits) % es) return SSD_ERR_ALIGN;
+    VerifyPlan plan;
+    int rc = plan_verify(B, M, V, dtype, opts, &plan);
+    if (rc != SSD_OK) return rc;
+    if (B > 0 && (!workspace || workspace_bytes < plan.workspace_bytes ||
+                  reinterpret_cast<uintptr_t>(workspace) % 256))
+        return SSD_ERR_WORKSPACE;
+    Launch L{static_cast<cudaStream_t>(stream), opts};
+    return launch_verify(logits, dtype, V, ld, M, tok_off, draft_ids, B, tau_slm, skip, workspace,
+                         token_logp, row_lse, accepted_len, all_accepted, utt_status, plan, L);
+}
+
+}  // extern "C"

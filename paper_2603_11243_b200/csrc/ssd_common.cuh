@@ -1,0 +1,236 @@
+// Shared device helpers of libssd: mbarrier / bulk-copy PTX wrappers for sm_100a, bounded
+// waits, logit unpacking and small warp reductions.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/ssd.h"
+
+namespace ssd {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr float kNegInit = -1.0e30f;          // "no value yet" for a running maximum
+constexpr long long kWaitLimitCycles = 1ll << 31;  // ~1 s at 2 GHz: bound of every spin wait
+
+// ---- host-side launch bookkeeping ----------------------------------------------------------
+struct Launch {
+    cudaStream_t stream;
+    const ssd_launch_opts *opts;
+};
+
+// ---- shared-memory addresses and mbarriers ---------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+
+// Makes freshly initialised barriers visible to the async (bulk-copy) proxy.
+__device__ __forceinline__ void mbar_init_fence() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+__device__ __forceinline__ void fence_proxy_async() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+                 : "memory");
+}
+
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
+
+// Waits for the phase with the given parity to complete, for at most kWaitLimitCycles.
+// Called by all 32 lanes of a warp; the answer is the same in every lane.  Returns false when
+// the limit ran out (the caller records the error and winds down).
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+    bool ok = mbar_try_wait(bar, parity);
+    if (!ok) {
+        const long long t0 = clock64();
+        while (!(ok = mbar_try_wait(bar, parity))) {
+            if (clock64() - t0 > kWaitLimitCycles) break;
+        }
+    }
+    return __all_sync(0xffffffffu, ok);
+}
+
+// 1-D bulk asynchronous copy global -> shared, completion counted in bytes on `bar`.
+// dst, src 16-byte aligned; bytes a positive multiple of 16.
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes,
+                                         uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+        : "memory");
+}
+
+// After a bounded wait has failed: give copies that may still be in flight time to land before
+// the CTA's shared memory is released (bounded as well).
+__device__ __forceinline__ void drain_after_error() {
+    const long long t0 = clock64();
+    while (clock64() - t0 < (1ll << 22)) __nanosleep(1000);
+}
+
+// ---- arithmetic -------------------------------------------------------------------------------
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// max of two packed bf16 pairs (NaN operands lose)
+__device__ __forceinline__ uint32_t bf16x2_max(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+
+// order-preserving map float -> int32 (for integer warp reductions of float maxima)
+__device__ __forceinline__ int32_t float_key(float f) {
+    int32_t b = __float_as_int(f);
+    return b >= 0 ? b : (b ^ 0x7fffffff);
+}
+__device__ __forceinline__ float key_float(int32_t k) {
+    return __int_as_float(k >= 0 ? k : (k ^ 0x7fffffff));
+}
+
+__device__ __forceinline__ float warp_max(float v) {
+    return key_float(__reduce_max_sync(0xffffffffu, float_key(v)));
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+template <typename T> struct Elem;
+template <> struct Elem<float> {
+    static constexpr int kBytes = 4;
+    static constexpr int kPerChunk = 4;  // elements in a 16-byte chunk
+    __device__ static __forceinline__ float load(const void *p) {
+        return *reinterpret_cast<const float *>(p);
+    }
+    __device__ static __forceinline__ float load_shared(uint32_t addr) {
+        float v;
+        asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+        return v;
+    }
+    static constexpr uint32_t kNegInfBits = 0xff800000u;
+};
+struct bf16_t { uint16_t bits; };
+template <> struct Elem<bf16_t> {
+    static constexpr int kBytes = 2;
+    static constexpr int kPerChunk = 8;
+    __device__ static __forceinline__ float load(const void *p) {
+        return __uint_as_float(static_cast<uint32_t>(*reinterpret_cast<const uint16_t *>(p)) << 16);
+    }
+    __device__ static __forceinline__ float load_shared(uint32_t addr) {
+        uint16_t v;
+        asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr));
+        return __uint_as_float(static_cast<uint32_t>(v) << 16);
+    }
+    static constexpr uint32_t kNegInfBits = 0xff80ff80u;
+};
+
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "r"(addr));
+    return v;
+}
+
+// maximum of the elements of one 16-byte chunk
+template <typename T> __device__ __forceinline__ float chunk_max(const uint4 &w);
+template <> __device__ __forceinline__ float chunk_max<float>(const uint4 &w) {
+    return fmaxf(fmaxf(__uint_as_float(w.x), __uint_as_float(w.y)),
+                 fmaxf(__uint_as_float(w.z), __uint_as_float(w.w)));
+}
+template <> __device__ __forceinline__ float chunk_max<bf16_t>(const uint4 &w) {
+    uint32_t h = bf16x2_max(bf16x2_max(w.x, w.y), bf16x2_max(w.z, w.w));
+    return fmaxf(bf16_lo(h), bf16_hi(h));
+}
+
+// element j of a 16-byte chunk as float
+template <typename T> __device__ __forceinline__ void chunk_unpack(const uint4 &w, float *x);
+template <> __device__ __forceinline__ void chunk_unpack<float>(const uint4 &w, float *x) {
+    x[0] = __uint_as_float(w.x); x[1] = __uint_as_float(w.y);
+    x[2] = __uint_as_float(w.z); x[3] = __uint_as_float(w.w);
+}
+template <> __device__ __forceinline__ void chunk_unpack<bf16_t>(const uint4 &w, float *x) {
+    x[0] = bf16_lo(w.x); x[1] = bf16_hi(w.x); x[2] = bf16_lo(w.y); x[3] = bf16_hi(w.y);
+    x[4] = bf16_lo(w.z); x[5] = bf16_hi(w.z); x[6] = bf16_lo(w.w); x[7] = bf16_hi(w.w);
+}
+
+// index b in [0,B) with off[b] <= r < off[b+1] for monotone offsets; stays inside [0,B) for
+// any offsets.  Returns -1 when B == 0.
+__device__ __forceinline__ int utterance_of_row(const int64_t *off, int B, int64_t r) {
+    if (B <= 0) return -1;
+    int lo = 0, hi = B - 1;
+    while (lo < hi) {
+        int mid = (lo + hi + 1) >> 1;
+        if (off[mid] <= r) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
+// ---- launchers implemented in the .cu files ---------------------------------------------------
+int launch_ctc_rows(const void *logits, ssd_dtype dtype, int V, int64_t ld, int64_t N,
+                    const int64_t *frame_off, int B, float *frame_entropy, int32_t *frame_argmax,
+                    float *frame_lse, float *frame_logprob, uint32_t *utt_status,
+                    const Launch &L);
+int launch_collapse(const int32_t *frame_argmax, const float *frame_entropy,
+                    const int64_t *frame_off, int B, int64_t N, int blank_id, int max_draft_len,
+                    int32_t *draft_tokens, int32_t *draft_frames, int32_t *draft_len,
+                    int32_t *draft_full_len, float *utt_max_entropy, uint32_t *utt_status,
+                    cudaStream_t stream);
+int launch_gate(const float *frame_entropy, const int64_t *frame_off, int B, int64_t N,
+                float tau, uint8_t *gate_accept, float *max_entropy, int32_t *argmax_frame,
+                cudaStream_t stream);
+
+struct VerifyPlan {
+    int kernel;        // 1 plain loads, 2 bulk-copy pipeline
+    int ctas;
+    int warps;         // consumer warps per CTA
+    int stages;
+    int stage_bytes;
+    int split;         // column spans per row
+    int partials;      // partial (max, sum) pairs per row = split * warps
+    size_t smem_bytes;
+    size_t workspace_bytes;
+};
+int plan_verify(int B, int64_t M, int V, ssd_dtype dtype, const ssd_launch_opts *opts,
+                VerifyPlan *plan);
+int launch_verify(const void *logits, ssd_dtype dtype, int V, int64_t ld, int64_t M,
+                  const int64_t *tok_off, const int32_t *draft_ids, int B, float tau_slm,
+                  const uint8_t *skip, void *workspace, float *token_logp, float *row_lse,
+                  int32_t *accepted_len, uint8_t *all_accepted, uint32_t *utt_status,
+                  const VerifyPlan &plan, const Launch &L);
+
+void record_cuda_error(cudaError_t e);
+
+}  // namespace ssd

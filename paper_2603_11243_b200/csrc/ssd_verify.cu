@@ -1,0 +1,488 @@
+// Stage 2 kernels: vocabulary-wide log-sum-exp of the LLM logits at the draft positions, the
+// draft token's log-likelihood (Eq. 5), and the first rejected position (Section 2.3).
+//
+// The LLM logits [M, V] are read once by a streaming kernel that leaves, for every row, a few
+// partial (max, sum-of-exponentials) pairs in the workspace; a small per-utterance kernel merges
+// them, gathers x[i, draft_i], applies the acceptance rule and finds the first reject.
+//
+//   verify_rows_tma    persistent CTAs; warp 0 is the producer: it walks this CTA's work items
+//                      (a row, or a column span of a row), and feeds a ring of shared-memory
+//                      stages with 1-D bulk asynchronous copies (TMA) signalled through
+//                      mbarriers.  The other warps consume: each thread keeps a running
+//                      reference maximum and a sum of 2^((x-m)*log2e), rescaling only when the
+//                      maximum moves by more than a fixed slack (so almost never), one
+//                      exponential per logit.
+//   verify_rows_plain  one CTA per item with scalar global loads; any alignment.  Fallback.
+#include <math.h>
+
+#include "ssd_common.cuh"
+
+namespace ssd {
+
+int device_sm_count();
+
+namespace {
+
+constexpr float kLazySlack = 8.0f;     // the running maximum may lag the true one by this much
+constexpr int kOffCacheMax = 2048;     // utterance offsets kept in shared memory up to this many
+constexpr uint32_t kFlagLast = 1u, kFlagEnd = 2u;
+
+struct VerifyParams {
+    const char *logits;
+    int V;
+    int64_t ld;
+    int64_t M;
+    int split;
+    int64_t num_items;
+    const int64_t *tok_off;
+    int B;
+    const uint8_t *skip;
+    float2 *partials;
+    int partials_per_row;
+    int warps;            // consumer warps
+    int stages;
+    int stage_bytes;
+    unsigned long long *err_word;
+    unsigned long long epoch;
+};
+
+struct StageDesc {
+    int32_t nchunks;
+    uint32_t flags;
+    int64_t slot;         // index of this item's first partial
+};
+
+struct Online {
+    float m, mh, S0, S1, S2, S3;
+    __device__ __forceinline__ void reset() {
+        m = kNegInit; mh = kNegInit * kLog2e; S0 = S1 = S2 = S3 = 0.f;
+    }
+    __device__ __forceinline__ void raise_to(float nm) {
+        const float sc = ex2(fmaf(m, kLog2e, -nm * kLog2e));
+        S0 *= sc; S1 *= sc; S2 *= sc; S3 *= sc;
+        m = nm; mh = nm * kLog2e;
+    }
+};
+
+template <typename T> __device__ __forceinline__ void consume_chunk(const uint4 &w, Online &st);
+template <> __device__ __forceinline__ void consume_chunk<float>(const uint4 &w, Online &st) {
+    const float cm = chunk_max<float>(w);
+    if (cm > st.m + kLazySlack) st.raise_to(cm);
+    st.S0 += ex2(fmaf(__uint_as_float(w.x), kLog2e, -st.mh));
+    st.S1 += ex2(fmaf(__uint_as_float(w.y), kLog2e, -st.mh));
+    st.S2 += ex2(fmaf(__uint_as_float(w.z), kLog2e, -st.mh));
+    st.S3 += ex2(fmaf(__uint_as_float(w.w), kLog2e, -st.mh));
+}
+template <> __device__ __forceinline__ void consume_chunk<bf16_t>(const uint4 &w, Online &st) {
+    const float cm = chunk_max<bf16_t>(w);
+    if (cm > st.m + kLazySlack) st.raise_to(cm);
+    st.S0 += ex2(fmaf(bf16_lo(w.x), kLog2e, -st.mh));
+    st.S1 += ex2(fmaf(bf16_hi(w.x), kLog2e, -st.mh));
+    st.S2 += ex2(fmaf(bf16_lo(w.y), kLog2e, -st.mh));
+    st.S3 += ex2(fmaf(bf16_hi(w.y), kLog2e, -st.mh));
+    st.S0 += ex2(fmaf(bf16_lo(w.z), kLog2e, -st.mh));
+    st.S1 += ex2(fmaf(bf16_hi(w.z), kLog2e, -st.mh));
+    st.S2 += ex2(fmaf(bf16_lo(w.w), kLog2e, -st.mh));
+    st.S3 += ex2(fmaf(bf16_hi(w.w), kLog2e, -st.mh));
+}
+
+// Warp-level merge of the lanes' (m, S) into one pair relative to the warp maximum.
+__device__ __forceinline__ float2 warp_merge(const Online &st) {
+    const float S = (st.S0 + st.S1) + (st.S2 + st.S3);
+    const float ml = fmaf(st.m, kLog2e, -st.mh);        // exponents carried +ml: take it out
+    const float M = warp_max(st.m);
+    // S == 0 covers lanes that saw nothing (their ml is meaningless); a NaN sum still propagates
+    const float Sw = warp_sum(S == 0.f ? 0.f : S * ex2(fmaf(st.m - M, kLog2e, -ml)));
+    return make_float2(M, Sw);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(544, 1) verify_rows_tma(const VerifyParams p) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    constexpr int ES = Elem<T>::kBytes, EPC = Elem<T>::kPerChunk;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int S = p.stages, CW = p.warps;
+    // layout: full[S] | empty[S] | desc[S] | offsets cache | stages
+    unsigned char *smem = reinterpret_cast<unsigned char *>(
+        (reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t full0 = sbase, empty0 = sbase + S * 8;
+    StageDesc *desc = reinterpret_cast<StageDesc *>(smem + 2 * S * 8);
+    const bool cache_off = p.skip != nullptr && p.B + 1 <= kOffCacheMax;
+    int64_t *off_cache = reinterpret_cast<int64_t *>(smem + 2 * S * 8 + S * sizeof(StageDesc));
+    const uint32_t hdr = (uint32_t)((2 * S * 8 + S * sizeof(StageDesc) +
+                                     (cache_off ? (size_t)(p.B + 1) * 8 : 0) + 127) & ~(size_t)127);
+    const uint32_t stage0 = sbase + hdr;
+    unsigned char *stage0_ptr = smem + hdr;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) { mbar_init(full0 + s * 8, 1); mbar_init(empty0 + s * 8, CW); }
+        mbar_init_fence();
+    }
+    if (cache_off)
+        for (int i = threadIdx.x; i <= p.B; i += blockDim.x) off_cache[i] = p.tok_off[i];
+    __syncthreads();
+
+    const int64_t row_bytes = (int64_t)p.V * ES;
+
+    if (warp == 0) {
+        // =============================== producer ===============================
+        const int64_t *offs = cache_off ? off_cache : p.tok_off;
+        int64_t it = 0;             // stages handed out so far
+        bool failed = false;
+        for (int64_t k0 = 0; !failed; k0 += 32) {
+            const int64_t first = (int64_t)blockIdx.x + k0 * gridDim.x;
+            if (first >= p.num_items) break;
+            const int64_t mine = first + (int64_t)lane * gridDim.x;
+            bool active = mine < p.num_items;
+            if (active && p.skip) {
+                const int b = utterance_of_row(offs, p.B, mine / p.split);
+                active = !(b >= 0 && p.skip[b]);
+            }
+            unsigned todo = __ballot_sync(0xffffffffu, active);
+            while (todo && !failed) {
+                const int src = __ffs(todo) - 1;
+                todo &= todo - 1;
+                const int64_t item = __shfl_sync(0xffffffffu, mine, src);
+                const int64_t row = item / p.split;
+                const int sp = (int)(item - row * p.split);
+                const uintptr_t g0 = reinterpret_cast<uintptr_t>(p.logits) +
+                                     (uintptr_t)(row * p.ld * ES);
+                const uintptr_t g1 = g0 + (uintptr_t)row_bytes;
+                const uintptr_t f0 = g0 & ~(uintptr_t)15;
+                const int64_t row_chunks = (int64_t)((((g1 + 15) & ~(uintptr_t)15) - f0) >> 4);
+                const int64_t cps = (row_chunks + p.split - 1) / p.split;
+                const int64_t sc0 = min(row_chunks, sp * cps), sc1 = min(row_chunks, sc0 + cps);
+                const int64_t span = sc1 - sc0;
+                const int64_t max_chunks = p.stage_bytes >> 4;
+                const int64_t parts = span > 0 ? (span + max_chunks - 1) / max_chunks : 1;
+                const int64_t per_part = span > 0 ? (span + parts - 1) / parts : 0;
+                const int64_t slot = row * p.partials_per_row + (int64_t)sp * CW;
+                for (int64_t part = 0; part < parts && !failed; ++part, ++it) {
+                    const int s = (int)(it % S);
+                    const uint32_t ph = (uint32_t)((it / S) & 1);
+                    if (!mbar_wait_bounded(empty0 + s * 8, ph ^ 1u)) { failed = true; break; }
+                    const int64_t pc0 = sc0 + part * per_part;
+                    const int64_t pc1 = min(sc1, pc0 + per_part);
+                    // chunks that are only partly inside the row (row start / end not on a
+                    // 16-byte boundary) are filled here with plain loads and -inf padding; the
+                    // bulk copy takes the fully valid chunks only, so it never leaves the row.
+                    int64_t b0 = pc0, b1 = pc1;
+                    unsigned char *dst = stage0_ptr + (size_t)s * p.stage_bytes;
+                    if (pc1 > pc0 && pc0 == 0 && f0 != g0) {
+                        b0 = 1;
+                        if (lane < EPC) {
+                            const uintptr_t a = f0 + (uintptr_t)lane * ES;
+                            const bool ok = a >= g0 && a < g1;
+                            if (ES == 4) reinterpret_cast<uint32_t *>(dst)[lane] =
+                                ok ? *reinterpret_cast<const uint32_t *>(a) : 0xff800000u;
+                            else reinterpret_cast<uint16_t *>(dst)[lane] =
+                                ok ? *reinterpret_cast<const uint16_t *>(a) : (uint16_t)0xff80u;
+                        }
+                    }
+                    if (pc1 > pc0 && pc1 == row_chunks && (g1 & 15) != 0 &&
+                        !(b0 == 1 && row_chunks == 1)) {
+                        b1 = pc1 - 1;
+                        if (lane < EPC) {
+                            const uintptr_t a = f0 + (uintptr_t)(pc1 - 1) * 16 + (uintptr_t)lane * ES;
+                            const bool ok = a >= g0 && a < g1;
+                            unsigned char *d = dst + (size_t)(pc1 - 1 - pc0) * 16;
+                            if (ES == 4) reinterpret_cast<uint32_t *>(d)[lane] =
+                                ok ? *reinterpret_cast<const uint32_t *>(a) : 0xff800000u;
+                            else reinterpret_cast<uint16_t *>(d)[lane] =
+                                ok ? *reinterpret_cast<const uint16_t *>(a) : (uint16_t)0xff80u;
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) {
+                        desc[s].nchunks = (int32_t)(pc1 - pc0);
+                        desc[s].flags = (part == parts - 1) ? kFlagLast : 0u;
+                        desc[s].slot = slot;
+                        const uint32_t bar = full0 + s * 8;
+                        if (b1 > b0) {
+                            const uint32_t bytes = (uint32_t)((b1 - b0) << 4);
+                            fence_proxy_async();
+                            mbar_arrive_expect_tx(bar, bytes);
+                            bulk_g2s(stage0 + (uint32_t)s * p.stage_bytes + (uint32_t)((b0 - pc0) << 4),
+                                     reinterpret_cast<const void *>(f0 + (uintptr_t)(b0 << 4)),
+                                     bytes, bar);
+                        } else {
+                            mbar_arrive(bar);
+                        }
+                    }
+                    __syncwarp();
+                }
+            }
+        }
+        if (!failed) {
+            const int s = (int)(it % S);
+            const uint32_t ph = (uint32_t)((it / S) & 1);
+            if (mbar_wait_bounded(empty0 + s * 8, ph ^ 1u)) {
+                if (lane == 0) {
+                    desc[s].nchunks = 0; desc[s].flags = kFlagEnd; desc[s].slot = 0;
+                    mbar_arrive(full0 + s * 8);
+                }
+            } else {
+                failed = true;
+            }
+        }
+        if (failed) {
+            if (lane == 0) atomicExch(p.err_word, p.epoch);
+            drain_after_error();
+        }
+    } else {
+        // =============================== consumers ===============================
+        const int cw = warp - 1;
+        const int ct = cw * 32 + lane, NT = CW * 32;
+        Online st;
+        st.reset();
+        bool failed = false;
+        for (int64_t it = 0;; ++it) {
+            const int s = (int)(it % S);
+            const uint32_t ph = (uint32_t)((it / S) & 1);
+            if (!mbar_wait_bounded(full0 + s * 8, ph)) { failed = true; break; }
+            const int n = desc[s].nchunks;
+            const uint32_t flags = desc[s].flags;
+            const int64_t slot = desc[s].slot;
+            if (flags & kFlagEnd) break;
+            const uint32_t a0 = stage0 + (uint32_t)s * p.stage_bytes;
+            int c = ct;
+            for (; c + 3 * NT < n; c += 4 * NT) {
+                const uint4 w0 = lds128(a0 + (uint32_t)c * 16);
+                const uint4 w1 = lds128(a0 + (uint32_t)(c + NT) * 16);
+                const uint4 w2 = lds128(a0 + (uint32_t)(c + 2 * NT) * 16);
+                const uint4 w3 = lds128(a0 + (uint32_t)(c + 3 * NT) * 16);
+                consume_chunk<T>(w0, st);
+                consume_chunk<T>(w1, st);
+                consume_chunk<T>(w2, st);
+                consume_chunk<T>(w3, st);
+            }
+            for (; c < n; c += NT) {
+                const uint4 w = lds128(a0 + (uint32_t)c * 16);
+                consume_chunk<T>(w, st);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty0 + s * 8);
+            if (flags & kFlagLast) {
+                const float2 r = warp_merge(st);
+                if (lane == 0) p.partials[slot + cw] = r;
+                st.reset();
+            }
+        }
+        if (failed) {
+            if (lane == 0) atomicExch(p.err_word, p.epoch);
+            drain_after_error();
+        }
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) verify_rows_plain(const VerifyParams p) {
+    constexpr int ES = Elem<T>::kBytes;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    for (int64_t item = blockIdx.x; item < p.num_items; item += gridDim.x) {
+        const int64_t row = item / p.split;
+        const int sp = (int)(item - row * p.split);
+        if (p.skip) {
+            const int b = utterance_of_row(p.tok_off, p.B, row);
+            if (b >= 0 && p.skip[b]) continue;
+        }
+        const int per = (p.V + p.split - 1) / p.split;
+        const int v0 = min(p.V, sp * per), v1 = min(p.V, v0 + per);
+        const char *rp = p.logits + row * p.ld * ES;
+        float m = kNegInit, S = 0.f;
+        for (int a = v0 + threadIdx.x; a < v1; a += blockDim.x) {
+            const float x = Elem<T>::load(rp + (size_t)a * ES);
+            if (x > m) { S = S * expf(m - x) + 1.f; m = x; }
+            else S += expf(x - m);
+        }
+        const float Mw = warp_max(m);
+        const float Sw = warp_sum(S * expf(m - Mw));
+        if (lane == 0) p.partials[row * p.partials_per_row + (int64_t)sp * nw + warp] =
+            make_float2(Mw, Sw);
+    }
+}
+
+constexpr int kFinishThreads = 256;
+
+template <typename T>
+__global__ void __launch_bounds__(kFinishThreads) verify_finish_kernel(
+    const char *__restrict__ logits, int V, int64_t ld, int64_t M,
+    const int64_t *__restrict__ tok_off, const int32_t *__restrict__ draft_ids, int B,
+    float log_tau, int reject_none, const uint8_t *__restrict__ skip,
+    const float2 *__restrict__ partials, int P, float *__restrict__ token_logp,
+    float *__restrict__ row_lse, int32_t *__restrict__ accepted_len,
+    uint8_t *__restrict__ all_accepted, uint32_t *__restrict__ utt_status,
+    const unsigned long long *err_word, unsigned long long epoch) {
+    constexpr int ES = Elem<T>::kBytes;
+    __shared__ int first_reject;
+    __shared__ unsigned flags;
+    const int b = blockIdx.x, tid = threadIdx.x;
+    const int64_t i0 = tok_off[b], i1 = tok_off[b + 1];
+    const uint32_t internal = (*err_word == epoch) ? (uint32_t)SSD_UTT_INTERNAL : 0u;
+    if (i0 < 0 || i1 < i0 || i1 > M) {
+        if (tid == 0) {
+            accepted_len[b] = 0; all_accepted[b] = 0;
+            utt_status[b] = SSD_UTT_BAD_OFFSETS | internal;
+        }
+        return;
+    }
+    const int64_t K64 = i1 - i0;
+    const int K = K64 > 0x7fffffff ? 0x7fffffff : (int)K64;
+    if (skip && skip[b]) {
+        if (tid == 0) { accepted_len[b] = K; all_accepted[b] = 1; utt_status[b] = internal; }
+        return;
+    }
+    if (tid == 0) { first_reject = K; flags = 0; }
+    __syncthreads();
+    unsigned myflags = 0;
+    int myfirst = K;
+    for (int i = tid; i < K; i += blockDim.x) {
+        const int64_t r = i0 + i;
+        const float2 *pp = partials + r * P;
+        float Mx = kNegInit;
+        for (int q = 0; q < P; ++q) Mx = fmaxf(Mx, pp[q].x);
+        float S = 0.f;
+        for (int q = 0; q < P; ++q) {
+            const float2 v = pp[q];
+            S += v.y * expf(v.x - Mx);
+        }
+        const float lse = Mx + logf(S);
+        if (!(fabsf(lse) < INFINITY)) myflags |= SSD_UTT_NONFINITE;
+        const int id = draft_ids[r];
+        float logp;
+        bool reject;
+        if (id < 0 || id >= V) {
+            myflags |= SSD_UTT_BAD_DRAFT_ID;
+            logp = -INFINITY;
+            reject = true;
+        } else {
+            const float x = Elem<T>::load(logits + (r * ld + id) * ES);
+            logp = x - lse;
+            reject = reject_none ? false : !(logp > log_tau);   // p <= tau; NaN rejects
+        }
+        token_logp[r] = logp;
+        if (row_lse) row_lse[r] = lse;
+        if (reject && i < myfirst) myfirst = i;
+    }
+    if (myfirst < K) atomicMin(&first_reject, myfirst);
+    if (myflags) atomicOr(&flags, myflags);
+    __syncthreads();
+    if (tid == 0) {
+        accepted_len[b] = first_reject;
+        all_accepted[b] = first_reject == K ? 1 : 0;
+        utt_status[b] = flags | internal;
+    }
+}
+
+}  // namespace
+
+unsigned long long next_epoch();
+
+// Workspace: [0,256) header (error word), then M * partials float2.
+int plan_verify(int B, int64_t M, int V, ssd_dtype dtype, const ssd_launch_opts *o,
+                VerifyPlan *plan) {
+    const int es = dtype == SSD_F32 ? 4 : 2;
+    VerifyPlan pl{};
+    pl.kernel = (o && o->kernel) ? o->kernel : 2;
+    if (pl.kernel != 1 && pl.kernel != 2) return SSD_ERR_ARG;
+    const int sms = device_sm_count();
+    pl.ctas = (o && o->ctas > 0) ? o->ctas : sms;
+    const int64_t row_bytes = (int64_t)V * es;
+    if (pl.kernel == 2) {
+        pl.warps = (o && o->warps > 0) ? o->warps : 8;
+        if (pl.warps > 16) return SSD_ERR_ARG;
+        pl.stage_bytes = (o && o->stage_bytes > 0) ? o->stage_bytes : 32768;
+        if (pl.stage_bytes < 1024 || pl.stage_bytes > 65536 || (pl.stage_bytes & 127))
+            return SSD_ERR_ARG;
+        const int off_cache = (B + 1 <= kOffCacheMax) ? (B + 1) * 8 : 0;
+        const int budget = 222 * 1024 - 512 - off_cache;
+        pl.stages = (o && o->stages > 0) ? o->stages : budget / pl.stage_bytes;
+        if (pl.stages > 16) pl.stages = 16;
+        if (pl.stages < 2 || (int64_t)pl.stages * pl.stage_bytes > budget) return SSD_ERR_ARG;
+        pl.smem_bytes = 128 + (size_t)((2 * pl.stages * 8 + pl.stages * sizeof(StageDesc) +
+                                        off_cache + 127) & ~127) +
+                        (size_t)pl.stages * pl.stage_bytes;
+    } else {
+        pl.warps = 8;
+        pl.stages = 0; pl.stage_bytes = 0; pl.smem_bytes = 0;
+    }
+    // column spans per row: enough items for a few balanced waves when there are few rows
+    int split = 1;
+    if (o && o->split > 0) {
+        split = o->split;
+    } else if (M > 0 && M < 8ll * pl.ctas) {
+        const int64_t want = (8ll * pl.ctas + M - 1) / M;
+        const int64_t most = row_bytes / 16384 > 1 ? row_bytes / 16384 : 1;  // spans >= 16 KB
+        split = (int)(want < most ? want : most);
+    }
+    if (split < 1) split = 1;
+    if (split > 64) split = 64;
+    pl.split = split;
+    pl.partials = split * pl.warps;
+    pl.workspace_bytes = 256 + (size_t)M * pl.partials * sizeof(float2);
+    *plan = pl;
+    return SSD_OK;
+}
+
+int launch_verify(const void *logits, ssd_dtype dtype, int V, int64_t ld, int64_t M,
+                  const int64_t *tok_off, const int32_t *draft_ids, int B, float tau_slm,
+                  const uint8_t *skip, void *workspace, float *token_logp, float *row_lse,
+                  int32_t *accepted_len, uint8_t *all_accepted, uint32_t *utt_status,
+                  const VerifyPlan &plan, const Launch &L) {
+    if (B == 0) return SSD_OK;
+    const ssd_launch_opts *o = L.opts;
+    unsigned long long *err_word = static_cast<unsigned long long *>(workspace);
+    float2 *partials = reinterpret_cast<float2 *>(static_cast<char *>(workspace) + 256);
+    const unsigned long long epoch = next_epoch();
+    cudaError_t e;
+    if (M > 0) {
+        VerifyParams p{};
+        p.logits = static_cast<const char *>(logits);
+        p.V = V; p.ld = ld; p.M = M; p.split = plan.split; p.num_items = M * plan.split;
+        p.tok_off = tok_off; p.B = B; p.skip = skip;
+        p.partials = partials; p.partials_per_row = plan.partials;
+        p.warps = plan.warps; p.stages = plan.stages; p.stage_bytes = plan.stage_bytes;
+        p.err_word = err_word; p.epoch = epoch;
+        int64_t ctas = p.num_items < plan.ctas ? p.num_items : plan.ctas;
+        if (o && o->ev_begin) {
+            e = cudaEventRecord(static_cast<cudaEvent_t>(o->ev_begin), L.stream);
+            if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
+        }
+        if (plan.kernel == 2) {
+            auto kern = dtype == SSD_F32 ? verify_rows_tma<float> : verify_rows_tma<bf16_t>;
+            e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)plan.smem_bytes);
+            if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
+            kern<<<(unsigned)ctas, (plan.warps + 1) * 32, plan.smem_bytes, L.stream>>>(p);
+        } else {
+            ctas = p.num_items < 8ll * plan.ctas ? p.num_items : 8ll * plan.ctas;
+            if (dtype == SSD_F32) verify_rows_plain<float><<<(unsigned)ctas, 256, 0, L.stream>>>(p);
+            else verify_rows_plain<bf16_t><<<(unsigned)ctas, 256, 0, L.stream>>>(p);
+        }
+        e = cudaGetLastError();
+        if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
+        if (o && o->ev_end) {
+            e = cudaEventRecord(static_cast<cudaEvent_t>(o->ev_end), L.stream);
+            if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
+        }
+    }
+    const double tau = (double)tau_slm;
+    const int reject_none = !(tau > 0.0);
+    const float log_tau = reject_none ? -INFINITY : (float)log(tau);
+    if (dtype == SSD_F32)
+        verify_finish_kernel<float><<<B, kFinishThreads, 0, L.stream>>>(
+            static_cast<const char *>(logits), V, ld, M, tok_off, draft_ids, B, log_tau,
+            reject_none, skip, partials, plan.partials, token_logp, row_lse, accepted_len,
+            all_accepted, utt_status, err_word, epoch);
+    else
+        verify_finish_kernel<bf16_t><<<B, kFinishThreads, 0, L.stream>>>(
+            static_cast<const char *>(logits), V, ld, M, tok_off, draft_ids, B, log_tau,
+            reject_none, skip, partials, plan.partials, token_logp, row_lse, accepted_len,
+            all_accepted, utt_status, err_word, epoch);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
+    return SSD_OK;
+}
+
+}  // namespace ssd

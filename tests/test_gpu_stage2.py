@@ -1,0 +1,185 @@
+"""GPU parity of stage 2 (ssd_verify) against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+import helpers as H
+from oracle import ref
+from paper_2603_11243_b200 import binding as ssd
+from paper_2603_11243_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+KERNELS = {"plain": 1, "tma": 2}
+
+
+def run_verify(logits_dev, tok_off, draft_ids, V, tau, skip=None, guard=True, **okw):
+    dev = logits_dev.device
+    M, B = logits_dev.shape[0], len(tok_off) - 1
+    o = H.opts(**okw)
+    code = ssd.BF16 if logits_dev.dtype == torch.bfloat16 else ssd.F32
+    ws = ssd.ssd_verify_workspace_bytes(B, M, V, code, o)
+    if guard:
+        g, out = H.guarded_verify_outputs(M, B, dev, ws)
+    else:
+        g, out = None, ssd.alloc_verify_outputs(M, B, dev, ws)
+    out["token_logp"].fill_(float("nan"))
+    skip_dev = None if skip is None else torch.as_tensor(skip, dtype=torch.uint8).to(dev)
+    ssd.ssd_verify(logits_dev, tok_off.to(dev), draft_ids.to(dev), tau, skip=skip_dev, V=V,
+                   out=out, opts=o)
+    torch.cuda.synchronize()
+    if g:
+        g.check()
+    return out
+
+
+def check_verify(w, K, device, kernel, skip=None, require_all_margins=True, **okw):
+    vb = synth.make_verify_batch(w, K, "cpu")
+    out = run_verify(vb.logits.to(device), vb.tok_off, vb.draft_ids, w.V_llm, w.tau_slm,
+                     skip=skip, kernel=kernel, **okw)
+    orc = ref.verify(H.storage_numpy(vb.logits), w.V_llm, vb.tok_off.numpy(),
+                     vb.draft_ids.numpy(), float(np.float32(w.tau_slm)), skip=skip)
+    H.compare_stage2(out, orc, vb.tok_off.numpy(), w.tau_slm, skip=skip,
+                     require_all_margins=require_all_margins)
+    return vb, out, orc
+
+
+@pytest.mark.parametrize("kernel", KERNELS.values(), ids=KERNELS.keys())
+def test_config0_tiny_planted_reject(cuda_device, kernel):
+    w = synth.CONFIGS[0]
+    vb, out, orc = check_verify(w, [37], cuda_device, kernel)
+    # anchored generator: the planted position is the first reject
+    assert int(orc["accepted_len"][0]) == int(vb.planted_reject[0])
+
+
+@pytest.mark.parametrize("kernel", KERNELS.values(), ids=KERNELS.keys())
+@pytest.mark.parametrize("variant", ["anchored", "literal"])
+def test_config1_reduced_batch(cuda_device, kernel, variant):
+    """Configuration 1's verify generator (V = 49,152 bf16) on 6 utterances of ragged length,
+    one of them empty."""
+    w = synth.scaled(synth.CONFIGS[1], B=6, variant=variant)
+    K = [23, 0, 57, 1, 40, 12]
+    vb, out, orc = check_verify(w, K, cuda_device, kernel,
+                                require_all_margins=(variant == "anchored"))
+    if variant == "anchored":
+        want = [int(p) if p >= 0 else k for p, k in zip(vb.planted_reject.tolist(), K)]
+        assert list(orc["accepted_len"]) == want
+        assert len(set(orc["all_accepted"])) == 2      # both outcomes occur
+
+
+@pytest.mark.parametrize("kernel", KERNELS.values(), ids=KERNELS.keys())
+def test_gate_skip_mask(cuda_device, kernel):
+    """Utterances the gate accepted are not read: their token_logp stays untouched."""
+    w = synth.scaled(synth.CONFIGS[2], B=5, V_llm=100352)
+    K = [9, 14, 3, 20, 6]
+    skip = np.array([1, 0, 1, 0, 0], np.uint8)
+    vb, out, orc = check_verify(w, K, cuda_device, kernel, skip=skip)
+    lp = out["token_logp"].cpu().numpy()
+    assert np.isnan(lp[:9]).all() and np.isnan(lp[23:26]).all() and not np.isnan(lp[9:23]).any()
+
+
+@pytest.mark.parametrize("kernel", KERNELS.values(), ids=KERNELS.keys())
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("V", [1, 2, 5, 8, 17, 1000, 4099, 32000, 50001, 152064])
+def test_vocabulary_sizes(cuda_device, kernel, dtype, V):
+    w = synth.scaled(synth.CONFIGS[1], B=3, V_llm=V, dtype=dtype, seed=200 + V % 97,
+                     variant="literal", tau_slm=0.1)
+    check_verify(w, [5, 9, 2], cuda_device, kernel, require_all_margins=False)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("split", [1, 2, 3, 7, 64])
+def test_column_spans(cuda_device, dtype, split):
+    """Rows cut into column spans (used when there are few rows): same results."""
+    w = synth.scaled(synth.CONFIGS[1], B=3, V_llm=49152 + 40, dtype=dtype, seed=31)
+    check_verify(w, [4, 7, 2], cuda_device, 2, split=split)
+    check_verify(w, [4, 7, 2], cuda_device, 1, split=split)
+
+
+@pytest.mark.parametrize("warps,stages,stage_bytes,ctas", [(4, 2, 4096, 3), (16, 3, 65536, 148),
+                                                            (8, 12, 16384, 7), (1, 16, 1024, 1)])
+def test_pipeline_shapes(cuda_device, warps, stages, stage_bytes, ctas):
+    w = synth.scaled(synth.CONFIGS[1], B=4, V_llm=32000, seed=17)
+    check_verify(w, [11, 3, 8, 5], cuda_device, 2, warps=warps, stages=stages,
+                 stage_bytes=stage_bytes, ctas=ctas)
+
+
+@pytest.mark.parametrize("kernel", KERNELS.values(), ids=KERNELS.keys())
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_padded_rows_and_misaligned_base(cuda_device, kernel, dtype):
+    """ld > V with a row pitch that is not a multiple of 16 bytes and a base that is only
+    element-aligned: rows start and end inside 16-byte chunks."""
+    V, ld = 5003, 5011
+    w = synth.scaled(synth.CONFIGS[1], B=3, V_llm=ld, dtype=dtype, seed=41, variant="literal")
+    vb = synth.make_verify_batch(w, [6, 1, 9], "cpu")
+    ids = (vb.draft_ids % V).to(torch.int32)
+    wide = vb.logits.to(cuda_device)
+    out = run_verify(wide[:, 5:5 + V], vb.tok_off, ids, V, 0.1, kernel=kernel)
+    orc = ref.verify(H.storage_numpy(vb.logits[:, 5:5 + V].contiguous()), V, vb.tok_off.numpy(),
+                     ids.numpy(), float(np.float32(0.1)))
+    H.compare_stage2(out, orc, vb.tok_off.numpy(), 0.1, require_all_margins=False)
+
+
+@pytest.mark.parametrize("kernel", KERNELS.values(), ids=KERNELS.keys())
+def test_bad_draft_ids_nonfinite_rows_and_thresholds(cuda_device, kernel):
+    V = 300
+    g = torch.Generator().manual_seed(8)
+    x = torch.randn((10, V), generator=g)
+    ids = torch.randint(0, V, (10,), generator=g, dtype=torch.int32)
+    for i in range(10):
+        x[i, ids[i]] += 12.0
+    off = torch.tensor([0, 3, 6, 10], dtype=torch.int64)
+    bad = ids.clone()
+    bad[4] = V          # utterance 1, position 1: out of range -> reject there, never read
+    bad[7] = -1         # utterance 2, position 1
+    x2 = x.clone()
+    x2[0, 3] = float("nan")   # utterance 0, row 0
+    x2[2, :10] = -float("inf")  # masked entries are fine
+    out = run_verify(x2.to(cuda_device), off, bad, V, 0.1, kernel=kernel)
+    st = H.status_u32(out["utt_status"])
+    assert st[0] == ssd.UTT_NONFINITE and st[1] == ssd.UTT_BAD_DRAFT_ID and st[2] == ssd.UTT_BAD_DRAFT_ID
+    assert list(out["accepted_len"].cpu().numpy()) == [0, 1, 1]
+    orc = ref.verify(x2.numpy(), V, off.numpy(), bad.numpy(), float(np.float32(0.1)))
+    np.testing.assert_array_equal(orc["accepted_len"], [0, 1, 1])
+    np.testing.assert_array_equal(st, orc["utt_status"] & 0xff)
+    # tau <= 0 rejects nothing, tau >= 1 everything
+    out0 = run_verify(x.to(cuda_device), off, ids, V, 0.0, kernel=kernel)
+    assert list(out0["accepted_len"].cpu().numpy()) == [3, 3, 4]
+    out1 = run_verify(x.to(cuda_device), off, ids, V, 1.0, kernel=kernel)
+    assert list(out1["accepted_len"].cpu().numpy()) == [0, 0, 0]
+
+
+@pytest.mark.parametrize("kernel", KERNELS.values(), ids=KERNELS.keys())
+def test_exact_threshold_is_a_reject(cuda_device, kernel):
+    """V = 2 with equal logits gives p = 0.5 exactly; with tau = 0.5 the position is rejected
+    (p <= tau), with the next float below 0.5 it is accepted."""
+    x = torch.zeros((3, 2), dtype=torch.float32)
+    ids = torch.tensor([0, 1, 0], dtype=torch.int32)
+    off = torch.tensor([0, 3], dtype=torch.int64)
+    out = run_verify(x.to(cuda_device), off, ids, 2, 0.5, kernel=kernel)
+    assert int(out["accepted_len"].cpu()[0]) == 0 and int(out["all_accepted"].cpu()[0]) == 0
+    below = float(np.nextafter(np.float32(0.5), np.float32(0)))
+    out = run_verify(x.to(cuda_device), off, ids, 2, below, kernel=kernel)
+    assert int(out["accepted_len"].cpu()[0]) == 3 and int(out["all_accepted"].cpu()[0]) == 1
+
+
+def test_empty_batch_and_malformed_offsets(cuda_device):
+    dev = cuda_device
+    x = torch.zeros((4, 9), dtype=torch.float32)
+    ids = torch.zeros(4, dtype=torch.int32)
+    out = run_verify(x[:0].to(dev), torch.zeros(1, dtype=torch.int64), ids[:0], 9, 0.1)
+    assert out["accepted_len"].numel() == 0
+    off = torch.tensor([0, 3, 2, 4], dtype=torch.int64)
+    out = run_verify(x.to(dev), off, ids, 9, 0.05)
+    st = H.status_u32(out["utt_status"])
+    assert st[1] == ssd.UTT_BAD_OFFSETS and int(out["all_accepted"].cpu()[1]) == 0
+
+
+def test_runs_are_bit_identical(cuda_device):
+    w = synth.scaled(synth.CONFIGS[1], B=4, seed=3)
+    vb = synth.make_verify_batch(w, [30, 11, 25, 8], "cpu")
+    x = vb.logits.to(cuda_device)
+    a = run_verify(x, vb.tok_off, vb.draft_ids, w.V_llm, 0.1, guard=False)
+    b = run_verify(x, vb.tok_off, vb.draft_ids, w.V_llm, 0.1, guard=False)
+    for k in ("token_logp", "row_lse", "accepted_len", "all_accepted"):
+        assert torch.equal(a[k], b[k]), k
