@@ -1,0 +1,483 @@
+#!/usr/bin/env python
+"""Benchmark of the draft-and-verify decision path (ssd_ctc_draft -> ssd_entropy_gate ->
+ssd_verify) on synthetic logits shaped like the paper's workloads.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+A step is one pass of the whole path over one ragged batch.  One JSON line is printed by rank 0:
+utterances/s with the inputs resident in HBM, the same metric end to end from pinned host
+buffers, the HBM roofline fraction of the dominant kernel (timed with CUDA events recorded by
+the library around that kernel), the clocks seen under load, and the CPU oracle timed on the
+host cores as a reported baseline.  `--impl reference` times that oracle alone.
+"""
+import argparse
+import datetime
+import hashlib
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "utterances/s for CTC draft+gate+verify"
+UNIT = "utterances/s"
+FALLBACK_HBM_GBS = 6650.0
+N_SETS = 3                      # distinct input batches rotated through, so no step finds its
+                                # inputs in the 126 MB L2
+TRAFFIC_FILE = os.path.join(ROOT, "paper_2603_11243_b200", "ncu_traffic.json")
+KERNEL_SOURCES = ["ssd_common.cuh", "ssd_ctc.cu", "ssd_verify.cu", "ssd_api.cu"]
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=1, help="workload index (1..3)")
+    ap.add_argument("--e2e-steps", type=int, default=30)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--ncu-small", action="store_true",
+                    help="profiling aid: one input set, no end-to-end leg, no CPU baseline")
+    return ap.parse_args()
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def kernel_source_hash() -> str:
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2603_11243_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def recorded_traffic(kernel: str, units: float):
+    """DRAM bytes per launch of `kernel` from the committed ncu capture, scaled by the units
+    (bytes of logits) this launch processes; None when the kernels changed since the capture."""
+    try:
+        with open(TRAFFIC_FILE) as f:
+            rec = json.load(f)
+        e = rec[kernel]
+        if rec.get("source_sha256") != kernel_source_hash():
+            return None
+        return float(e["dram_bytes_per_launch"]) * units / float(e["algorithmic_bytes_per_launch"])
+    except Exception:
+        return None
+
+
+# ---- clocks --------------------------------------------------------------------------------
+CLOCK_FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+                "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+                "clocks_event_reasons.sw_power_cap")
+
+
+class ClockSampler:
+    def __init__(self, device_index: int):
+        import torch
+        self.path = tempfile.mktemp(prefix="ssd_clocks_", suffix=".csv")
+        uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+        if not uuid.startswith("GPU-"):
+            uuid = "GPU-" + uuid
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "--id=" + uuid, "--query-gpu=" + CLOCK_FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "50"],
+                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except OSError:
+            pass
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        rows = []
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 8:
+                    continue
+                try:
+                    ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                    rows.append((ts, float(f[1]), float(f[2]), f[4:8]))
+                except ValueError:
+                    continue
+            os.unlink(self.path)
+        except OSError:
+            pass
+        return rows
+
+
+def summarise_clocks(rows, windows, note):
+    names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+    inside = [r for r in rows if any(a <= r[0] <= b for a, b in windows)]
+    if not inside:
+        return {"sm_mhz": None, "sm_max_mhz": rows[0][2] if rows else None, "reasons": [],
+                "samples": 0, "note": "no nvidia-smi sample fell inside the load windows"}
+    reasons = sorted({n for r in inside for n, v in zip(names, r[3]) if v == "Active"})
+    return {"sm_mhz": statistics.median(r[1] for r in inside), "sm_max_mhz": inside[0][2],
+            "reasons": reasons, "samples": len(inside), "note": note}
+
+
+# ---- our arm ---------------------------------------------------------------------------------
+def build_sets(w, device, n_sets):
+    """Input sets and pre-marshalled calls.  The verify logits of a set have one row per draft
+    token of the set's own CTC drafts (found by running stage 1 once, untimed)."""
+    import torch
+    from paper_2603_11243_b200 import binding as ssd
+    from paper_2603_11243_b200 import synth
+    sets = []
+    for i in range(n_sets):
+        wi = synth.scaled(w, seed=w.seed + 7 * i)
+        cb = synth.make_ctc_batch(wi, device)
+        B, N = wi.B, cb.logits.shape[0]
+        off = cb.frame_off.to(device)
+        s1 = ssd.alloc_ctc_outputs(N, B, device)
+        ssd.ssd_ctc_draft(cb.logits, off, wi.blank_id, wi.max_draft_len, out=s1)
+        gate = ssd.alloc_gate_outputs(B, device)
+        ssd.ssd_entropy_gate(s1["frame_entropy"], off, wi.tau_ctc, out=gate)
+        torch.cuda.synchronize()
+        K = s1["draft_len"].cpu().tolist()
+        vb = synth.make_verify_batch(wi, K, device)
+        M = vb.logits.shape[0]
+        tok_off, ids = vb.tok_off.to(device), vb.draft_ids.to(device)
+        code = ssd.BF16 if wi.dtype == "bf16" else ssd.F32
+        s2 = ssd.alloc_verify_outputs(M, B, device, ssd.ssd_verify_workspace_bytes(B, M, wi.V_llm, code))
+        skipped = gate["gate_accept"].cpu().numpy().astype(bool)
+        m_active = int(sum(k for k, s in zip(K, skipped) if not s))
+        es = 2 if wi.dtype == "bf16" else 4
+        sets.append(dict(
+            w=wi, cb=cb, vb=vb, off=off, tok_off=tok_off, ids=ids, s1=s1, gate=gate, s2=s2,
+            B=B, N=N, M=M, K=K, m_active=m_active,
+            ctc_bytes=N * wi.V_ctc * es, verify_bytes=m_active * wi.V_llm * es,
+            call_ctc=ssd.bind_ctc_draft(cb.logits, off, wi.blank_id, wi.max_draft_len, s1),
+            call_gate=ssd.bind_entropy_gate(s1["frame_entropy"], off, wi.tau_ctc, gate),
+            call_verify=ssd.bind_verify(vb.logits, tok_off, ids, wi.tau_slm, s2,
+                                        skip=gate["gate_accept"])))
+    return sets
+
+
+def make_events(n):
+    """n timing events whose CUDA handles exist (torch creates the handle at the first record)."""
+    import torch
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+    for e in evs:
+        e.record()
+    torch.cuda.synchronize()
+    return evs
+
+
+def run_ours(args):
+    import torch
+    from paper_2603_11243_b200 import binding as ssd
+    from paper_2603_11243_b200 import build as lib_build
+    from paper_2603_11243_b200 import dist as D
+    from paper_2603_11243_b200 import synth
+
+    rank, local_rank, world = D.init("nccl")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: libssd has no CPU path")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if rank == 0:
+        lib_build.build()
+    D.barrier()
+    ssd.lib()
+
+    base = synth.CONFIGS[args.config]
+    w = synth.scaled(base, seed=D.rank_seed(base.seed, rank))
+    n_sets = 1 if args.ncu_small else N_SETS
+    sets = build_sets(w, device, n_sets)
+    K, W = args.steps, args.warmup
+
+    def step(s, o_ctc=None, o_ver=None):
+        s["call_ctc"](o_ctc)
+        s["call_gate"]()
+        s["call_verify"](o_ver)
+
+    for i in range(W):
+        step(sets[i % n_sets])
+    torch.cuda.synchronize()
+
+    # ---- timed region: K steps, inputs resident in HBM -------------------------------------
+    ev = make_events(4 * K + 2)
+    opts_ctc, opts_ver = [], []
+    for i in range(K):
+        a, b = ssd.LaunchOpts(), ssd.LaunchOpts()
+        a.ev_begin, a.ev_end = ev[4 * i].cuda_event, ev[4 * i + 1].cuda_event
+        b.ev_begin, b.ev_end = ev[4 * i + 2].cuda_event, ev[4 * i + 3].cuda_event
+        opts_ctc.append(a)
+        opts_ver.append(b)
+    t_begin, t_end = ev[4 * K], ev[4 * K + 1]
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    D.barrier()
+    torch.cuda.synchronize()
+    wall0 = time.time()
+    t_begin.record()
+    for i in range(K):
+        step(sets[i % n_sets], opts_ctc[i], opts_ver[i])
+    t_end.record()
+    torch.cuda.synchronize()
+    wall1 = time.time()
+    D.barrier()
+    ms_total = t_begin.elapsed_time(t_end)
+    windows, clock_note = [(wall0, wall1)], "timed region"
+    if rank == 0 and wall1 - wall0 < 0.6:
+        # the region is too short for a 50 ms sampler: keep the same load up a little longer
+        wall2 = time.time()
+        i = 0
+        while time.time() - wall2 < 0.7:
+            step(sets[i % n_sets])
+            i += 1
+            if i % 50 == 0:
+                torch.cuda.synchronize()
+        torch.cuda.synchronize()
+        windows.append((wall2, time.time()))
+        clock_note = "timed region plus %d further untimed steps of the same load" % i
+    clock_rows = sampler.stop() if sampler else []
+
+    ms_max, units = D.reduce_max_sum(ms_total, float(sum(sets[i % n_sets]["B"] for i in range(K))),
+                                     device)
+    value = units / (ms_max * 1e-3)
+
+    t_ctc = [ev[4 * i].elapsed_time(ev[4 * i + 1]) for i in range(K)]
+    t_ver = [ev[4 * i + 2].elapsed_time(ev[4 * i + 3]) for i in range(K)]
+    ctc_bytes = statistics.mean(sets[i % n_sets]["ctc_bytes"] for i in range(K))
+    ver_bytes = statistics.mean(sets[i % n_sets]["verify_bytes"] for i in range(K))
+    peak, peak_kind = peaks()
+
+    def roof(kernel, nbytes, times_ms):
+        avg = statistics.mean(times_ms)
+        ach = nbytes / (avg * 1e-3) / 1e9 if avg > 0 else 0.0
+        return {"kernel": kernel, "bound": "hbm", "achieved": round(ach, 1), "peak": peak,
+                "unit": "GB/s", "frac": round(ach / peak, 4), "peak_kind": "of " + peak_kind,
+                "traffic": recorded_traffic(kernel, nbytes),
+                "algorithmic_bytes_per_launch": int(nbytes),
+                "avg_launch_us": round(avg * 1e3, 2), "min_launch_us": round(min(times_ms) * 1e3, 2)}
+
+    # ---- end to end: pinned host buffers in, decisions out, every step ---------------------
+    e2e = None
+    if not args.ncu_small:
+        e2e = run_e2e(sets[0], device, args.e2e_steps, D, world)
+
+    if rank != 0:
+        D.finalize()
+        return
+    s0 = sets[0]
+    gate_acc = float(s0["gate"]["gate_accept"].float().mean().item())
+    all_acc = s0["s2"]["all_accepted"].cpu().numpy().astype(bool)
+    skipped = s0["gate"]["gate_accept"].cpu().numpy().astype(bool)
+    line = {
+        "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": K,
+        "warmup": W, "ms_per_step": round(ms_max / K, 5), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {
+            "workload": "configs[%d] %s: B=%d utterances per GPU, T~%s[%d,%d], V_ctc=%d, "
+                        "V_llm=%d, draft_len<=%d, %s logits (fp32 accumulation)" %
+                        (args.config, base.name, w.B, w.t_dist, w.t_lo, w.t_hi, w.V_ctc, w.V_llm,
+                         w.max_draft_len, w.dtype),
+            "generator": w.variant, "tau_ctc": w.tau_ctc, "tau_slm": w.tau_slm,
+            "frames_per_step": s0["N"], "verify_rows_per_step": s0["M"],
+            "verify_rows_read_per_step": s0["m_active"],
+            "logits_bytes_per_step": int(ctc_bytes + ver_bytes),
+            "l2": "inputs larger than L2: %d distinct input batches of %.2f GB rotated, each "
+                  "step reads %.2f GB once" % (n_sets, (s0["ctc_bytes"] + s0["M"] * w.V_llm * 2) / 1e9,
+                                              (ctc_bytes + ver_bytes) / 1e9),
+            "parallelism": "utterances sharded over %d rank(s), no data-path collective" % world},
+        "gpu_launches": 5 * K,
+        "roofline": roof("verify_rows_tma", ver_bytes, t_ver),
+        "roofline_ctc": roof("ctc_rows_tma", ctc_bytes, t_ctc),
+        "step_hbm_gbs": round((ctc_bytes + ver_bytes) / (ms_max / K * 1e-3) / 1e9, 1),
+        "step_frac_of_peak": round((ctc_bytes + ver_bytes) / (ms_max / K * 1e-3) / 1e9 / peak, 4),
+        "decisions": {"gate_accept_frac": round(gate_acc, 4),
+                      "verify_all_accepted_frac_of_verified":
+                          round(float(all_acc[~skipped].mean()) if (~skipped).any() else 0.0, 4)},
+        "clocks": summarise_clocks(clock_rows, windows, clock_note),
+        "e2e": e2e,
+    }
+    if world == 1 and not args.no_cpu_baseline and not args.ncu_small:
+        line["cpu_baseline"] = cpu_baseline(s0, budget_s=12.0)
+    print(json.dumps(line), flush=True)
+    D.finalize()
+
+
+def run_e2e(s, device, steps, D, world):
+    """The same path through the public binding with every input starting in pinned host
+    memory: each step copies the logits, offsets and draft ids to the device, makes the three
+    calls and reads the per-utterance decisions and the draft back to the host."""
+    import torch
+    w = s["w"]
+    pin = lambda t: t.detach().cpu().contiguous().pin_memory()
+    h_in = dict(ctc=pin(s["cb"].logits), llm=pin(s["vb"].logits), off=pin(s["off"]),
+                tok_off=pin(s["tok_off"]), ids=pin(s["ids"]))
+    d_in = dict(ctc=s["cb"].logits, llm=s["vb"].logits, off=s["off"], tok_off=s["tok_off"],
+                ids=s["ids"])
+    outs = [s["s1"]["draft_tokens"], s["s1"]["draft_len"], s["s1"]["utt_max_entropy"],
+            s["gate"]["gate_accept"], s["s2"]["accepted_len"], s["s2"]["all_accepted"],
+            s["s2"]["token_logp"], s["s1"]["utt_status"], s["s2"]["utt_status"]]
+    h_out = [torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in outs]
+    h2d = sum(t.numel() * t.element_size() for t in h_in.values())
+    d2h = sum(t.numel() * t.element_size() for t in outs)
+
+    def one():
+        for k in h_in:
+            d_in[k].copy_(h_in[k], non_blocking=True)
+        s["call_ctc"]()
+        s["call_gate"]()
+        s["call_verify"]()
+        for d, h in zip(outs, h_out):
+            h.copy_(d, non_blocking=True)
+        torch.cuda.current_stream().synchronize()      # the caller reads the decisions now
+
+    for _ in range(3):
+        one()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    D.barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    e0.record()
+    for _ in range(steps):
+        one()
+    e1.record()
+    torch.cuda.synchronize()
+    wall = time.perf_counter() - t0
+    D.barrier()
+    # host waits are part of this number: take the larger of device and wall time
+    sec = max(e0.elapsed_time(e1) * 1e-3, wall)
+    sec_max, units = D.reduce_max_sum(sec, float(steps * s["B"]), device)
+    return {"value": round(units / sec_max, 1), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+            "d2h_bytes_per_step": int(d2h), "steps": steps,
+            "ms_per_step": round(sec_max / steps * 1e3, 4),
+            "note": "pinned host -> device copies of all logits, three C-ABI calls, decisions "
+                    "and draft copied back, stream synchronised every step"}
+
+
+# ---- the oracle as a CPU baseline ------------------------------------------------------------
+def host_inputs(s):
+    import numpy as np
+    import torch
+
+    def to_np(t):
+        t = t.detach().cpu().contiguous()
+        if t.dtype == torch.bfloat16:
+            return t.view(torch.int16).numpy().view(np.uint16)
+        return t.numpy()
+    return dict(ctc=to_np(s["cb"].logits), llm=to_np(s["vb"].logits),
+                off=s["cb"].frame_off.numpy(), tok_off=s["vb"].tok_off.numpy(),
+                ids=s["vb"].draft_ids.numpy())
+
+
+def oracle_pass(h, w, lo, hi):
+    """The oracle's whole path on utterances [lo, hi) of a host batch; returns seconds."""
+    import numpy as np
+    from oracle import ref
+    off, tok = h["off"], h["tok_off"]
+    f0, f1, k0, k1 = int(off[lo]), int(off[hi]), int(tok[lo]), int(tok[hi])
+    t0 = time.perf_counter()
+    o1 = ref.ctc_draft(h["ctc"][f0:f1], w.V_ctc, off[lo:hi + 1] - f0, w.blank_id, w.max_draft_len)
+    g = ref.entropy_gate(o1["frame_entropy"], off[lo:hi + 1] - f0, float(np.float32(w.tau_ctc)))
+    ref.verify(h["llm"][k0:k1], w.V_llm, tok[lo:hi + 1] - k0, h["ids"][k0:k1],
+               float(np.float32(w.tau_slm)), skip=g["gate_accept"])
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(s, budget_s):
+    from oracle import ref
+    w = s["w"]
+    cores = len(os.sched_getaffinity(0))
+    threads = ref.set_threads(max(1, min(cores, w.B)))
+    h = host_inputs(s)
+    t1 = oracle_pass(h, w, 0, min(w.B, threads))            # one utterance per thread
+    per_utt = t1 / min(w.B, threads)
+    n = int(max(threads, min(w.B, budget_s / max(per_utt, 1e-9))))
+    n = min(w.B, n)
+    sec = oracle_pass(h, w, 0, n)
+    return {"value": round(n / sec, 2), "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": "first %d of the %d utterances of one configs[*] batch, whole path "
+                      "(fp64 two-pass C oracle, one utterance per thread), %.1f s" % (n, w.B, sec)}
+
+
+def run_reference(args):
+    """Times the CPU oracle on this arm's workload; rank 0 only."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import torch
+    from oracle import ref
+    from paper_2603_11243_b200 import synth
+    w = synth.CONFIGS[args.config]
+    K, W = args.steps, args.warmup
+    dev = "cpu"
+    cb = synth.make_ctc_batch(w, dev)
+    # the oracle's own drafts size the verify batch, as the GPU arm's drafts size its batch
+    import numpy as np
+    def to_np(t):
+        t = t.contiguous()
+        return t.view(torch.int16).numpy().view(np.uint16) if t.dtype == torch.bfloat16 else t.numpy()
+    ctc = to_np(cb.logits)
+    cores = len(os.sched_getaffinity(0))
+    threads = ref.set_threads(max(1, min(cores, w.B)))
+    o1 = ref.ctc_draft(ctc, w.V_ctc, cb.frame_off.numpy(), w.blank_id, w.max_draft_len)
+    vb = synth.make_verify_batch(w, o1["draft_len"].tolist(), dev)
+    h = dict(ctc=ctc, llm=to_np(vb.logits), off=cb.frame_off.numpy(), tok_off=vb.tok_off.numpy(),
+             ids=vb.draft_ids.numpy())
+    # bounded sample per step: u utterances, sized so that K + W steps take about two minutes
+    probe = oracle_pass(h, w, 0, min(w.B, threads)) / min(w.B, threads)
+    u = int(max(1, min(w.B, 120.0 / max(K + W, 1) / max(probe, 1e-9))))
+    starts = [(i * u) % max(1, w.B - u + 1) for i in range(K + W)]
+    for i in range(W):
+        oracle_pass(h, w, starts[i], starts[i] + u)
+    t0 = time.perf_counter()
+    for i in range(W, W + K):
+        oracle_pass(h, w, starts[i], starts[i] + u)
+    sec = time.perf_counter() - t0
+    value = K * u / sec
+    sample = ("%d utterance(s) of the configs[%d] batch per step (window sliding over the batch), "
+              "whole path in the fp64 C oracle, %d thread(s)" % (u, args.config, threads))
+    line = {"impl": "reference", "metric": METRIC, "value": round(value, 3), "unit": UNIT,
+            "n_gpus": args.gpus, "steps": K, "warmup": W, "ms_per_step": round(sec / K * 1e3, 3),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic",
+            "config": {"workload": "configs[%d] %s (CPU oracle on a bounded sample per step)" %
+                                   (args.config, w.name), "sample": sample},
+            "cpu_baseline": {"value": round(value, 3), "unit": UNIT, "cores": threads,
+                             "kind": "oracle", "sample": sample},
+            "e2e": {"value": round(value, 3), "unit": UNIT, "h2d_bytes_per_step": 0,
+                    "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1",
+               "--nproc-per-node", str(args.gpus), "--master-addr", "127.0.0.1",
+               "--master-port", "29533", os.path.abspath(__file__)] + sys.argv[1:]
+        raise SystemExit(subprocess.call(cmd))
+    run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

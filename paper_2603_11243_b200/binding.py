@@ -7,7 +7,7 @@ module without a built libssd.so, or calling it with host tensors, raises.
 """
 import ctypes as C
 import os
-from typing import Dict, Optional
+from typing import Callable, Dict, List, Optional
 
 import torch
 
@@ -201,3 +201,64 @@ def ssd_verify(logits: torch.Tensor, tok_off: torch.Tensor, draft_ids: torch.Ten
     if rc != OK:
         raise SsdError(rc, "ssd_verify")
     return out
+
+
+class BoundCall:
+    """One C-ABI call with its arguments already marshalled, for loops that issue the same call
+    many times (benchmarks, serving loops): calling it enqueues the work again on the stream
+    that was current when it was bound.  `opts` replaces the launch options for one call."""
+
+    def __init__(self, fn, name: str, args: List, keep: tuple, has_opts: bool):
+        self._fn, self._name, self._args, self._keep, self._has_opts = fn, name, args, keep, has_opts
+
+    def __call__(self, opts: Optional[LaunchOpts] = None) -> None:
+        a = self._args
+        if opts is not None:
+            if not self._has_opts:
+                raise TypeError(self._name + " takes no launch options")
+            a = a[:-1] + [C.cast(C.pointer(opts), C.c_void_p)]
+        rc = self._fn(*a)
+        if rc != OK:
+            raise SsdError(rc, self._name)
+
+
+def bind_ctc_draft(logits, frame_off, blank_id, max_draft_len, out, V=None,
+                   opts: Optional[LaunchOpts] = None) -> BoundCall:
+    N, ld = _rows_ld(logits)
+    V = logits.shape[1] if V is None else V
+    B = frame_off.shape[0] - 1
+    args = [_dev(logits, "logits"), _dtype_code(logits), V, ld, _dev(frame_off, "frame_off"), B, N,
+            blank_id, max_draft_len, _dev(out["frame_entropy"], "frame_entropy"),
+            _dev(out["frame_argmax"], "frame_argmax"), _dev(out.get("frame_lse"), "frame_lse"),
+            None, _dev(out["draft_tokens"], "draft_tokens"),
+            _dev(out.get("draft_frames"), "draft_frames"), _dev(out["draft_len"], "draft_len"),
+            _dev(out["draft_full_len"], "draft_full_len"),
+            _dev(out["utt_max_entropy"], "utt_max_entropy"), _dev(out["utt_status"], "utt_status"),
+            None, 0, _stream(), _opts(opts)]
+    return BoundCall(lib().ssd_ctc_draft, "ssd_ctc_draft", args, (logits, frame_off, out, opts), True)
+
+
+def bind_entropy_gate(frame_entropy, frame_off, tau_ctc, out) -> BoundCall:
+    B, N = frame_off.shape[0] - 1, frame_entropy.shape[0]
+    args = [_dev(frame_entropy, "frame_entropy"), _dev(frame_off, "frame_off"), B, N,
+            C.c_float(tau_ctc), _dev(out["gate_accept"], "gate_accept"),
+            _dev(out["max_entropy"], "max_entropy"), _dev(out.get("argmax_frame"), "argmax_frame"),
+            _stream()]
+    return BoundCall(lib().ssd_entropy_gate, "ssd_entropy_gate", args,
+                     (frame_entropy, frame_off, out), False)
+
+
+def bind_verify(logits, tok_off, draft_ids, tau_slm, out, skip=None, V=None,
+                opts: Optional[LaunchOpts] = None) -> BoundCall:
+    M, ld = _rows_ld(logits)
+    V = logits.shape[1] if V is None else V
+    B = tok_off.shape[0] - 1
+    ws = out["workspace"]
+    args = [_dev(logits, "logits"), _dtype_code(logits), V, ld, _dev(tok_off, "tok_off"),
+            _dev(draft_ids, "draft_ids"), B, M, C.c_float(tau_slm), _dev(skip, "skip"),
+            _dev(out["token_logp"], "token_logp"), _dev(out.get("row_lse"), "row_lse"),
+            _dev(out["accepted_len"], "accepted_len"), _dev(out["all_accepted"], "all_accepted"),
+            _dev(out["utt_status"], "utt_status"), _dev(ws, "workspace"), ws.numel(), _stream(),
+            _opts(opts)]
+    return BoundCall(lib().ssd_verify, "ssd_verify", args,
+                     (logits, tok_off, draft_ids, out, skip, opts), True)
