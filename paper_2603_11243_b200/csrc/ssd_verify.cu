@@ -8,10 +8,10 @@
 //   verify_rows_tma    persistent CTAs; warp 0 is the producer: it walks this CTA's work items
 //                      (a row, or a column span of a row), and feeds a ring of shared-memory
 //                      stages with 1-D bulk asynchronous copies (TMA) signalled through
-//                      mbarriers.  The other warps consume: each thread keeps a running
-//                      reference maximum and a sum of 2^((x-m)*log2e), rescaling only when the
-//                      maximum moves by more than a fixed slack (so almost never), one
-//                      exponential per logit.
+//                      mbarriers.  The other warps consume: each thread keeps a sum of
+//                      2^((x-m)*log2e) relative to a reference logit m of its own and checks
+//                      once per stage that the sum stayed in range (see Online), so the common
+//                      case is one exponential and no comparison per logit.
 //   verify_rows_plain  one CTA per item with scalar global loads; any alignment.  Fallback.
 #include <math.h>
 
@@ -23,9 +23,9 @@ int device_sm_count();
 
 namespace {
 
-constexpr float kLazySlack = 8.0f;     // the running maximum may lag the true one by this much
 constexpr int kOffCacheMax = 2048;     // utterance offsets kept in shared memory up to this many
 constexpr uint32_t kFlagLast = 1u, kFlagEnd = 2u;
+constexpr float kSumLimit = 1.0e30f;   // a running sum at or above this (or NaN) is recomputed
 
 struct VerifyParams {
     const char *logits;
@@ -52,46 +52,94 @@ struct StageDesc {
     int64_t slot;         // index of this item's first partial
 };
 
+// Running sum of exponentials of one thread, relative to a reference logit m that is one of the
+// thread's own elements (or -inf while it has seen none).  fp32 keeps full relative precision
+// over its whole exponent range, so m need not be the maximum: a thread only has to notice when
+// a sum came near overflow (an element far above m), which it does once per stage, and then
+// redoes that stage from shared memory with the proper maximum.  The common case therefore
+// costs one exponential and no comparison per logit.
 struct Online {
-    float m, mh, S0, S1, S2, S3;
+    float m, mh;
+    float2 Sa, Sb;
     __device__ __forceinline__ void reset() {
-        m = kNegInit; mh = kNegInit * kLog2e; S0 = S1 = S2 = S3 = 0.f;
+        m = -INFINITY; mh = -INFINITY; Sa = Sb = make_float2(0.f, 0.f);
     }
+    __device__ __forceinline__ float total() const { return (Sa.x + Sa.y) + (Sb.x + Sb.y); }
     __device__ __forceinline__ void raise_to(float nm) {
-        const float sc = ex2(fmaf(m, kLog2e, -nm * kLog2e));
-        S0 *= sc; S1 *= sc; S2 *= sc; S3 *= sc;
+        const float sc = ex2(fmaf(m, kLog2e, -nm * kLog2e));      // 0 when m is still -inf
+        Sa = fmul2(Sa, make_float2(sc, sc));
+        Sb = fmul2(Sb, make_float2(sc, sc));
         m = nm; mh = nm * kLog2e;
     }
 };
 
-template <typename T> __device__ __forceinline__ void consume_chunk(const uint4 &w, Online &st);
-template <> __device__ __forceinline__ void consume_chunk<float>(const uint4 &w, Online &st) {
-    const float cm = chunk_max<float>(w);
-    if (cm > st.m + kLazySlack) st.raise_to(cm);
-    st.S0 += ex2(fmaf(__uint_as_float(w.x), kLog2e, -st.mh));
-    st.S1 += ex2(fmaf(__uint_as_float(w.y), kLog2e, -st.mh));
-    st.S2 += ex2(fmaf(__uint_as_float(w.z), kLog2e, -st.mh));
-    st.S3 += ex2(fmaf(__uint_as_float(w.w), kLog2e, -st.mh));
+__device__ __forceinline__ float2 exp2_pair(float2 x, float2 scale, float2 nmh) {
+    const float2 t = ffma2(x, scale, nmh);
+    return make_float2(ex2(t.x), ex2(t.y));
 }
-template <> __device__ __forceinline__ void consume_chunk<bf16_t>(const uint4 &w, Online &st) {
-    const float cm = chunk_max<bf16_t>(w);
-    if (cm > st.m + kLazySlack) st.raise_to(cm);
-    st.S0 += ex2(fmaf(bf16_lo(w.x), kLog2e, -st.mh));
-    st.S1 += ex2(fmaf(bf16_hi(w.x), kLog2e, -st.mh));
-    st.S2 += ex2(fmaf(bf16_lo(w.y), kLog2e, -st.mh));
-    st.S3 += ex2(fmaf(bf16_hi(w.y), kLog2e, -st.mh));
-    st.S0 += ex2(fmaf(bf16_lo(w.z), kLog2e, -st.mh));
-    st.S1 += ex2(fmaf(bf16_hi(w.z), kLog2e, -st.mh));
-    st.S2 += ex2(fmaf(bf16_lo(w.w), kLog2e, -st.mh));
-    st.S3 += ex2(fmaf(bf16_hi(w.w), kLog2e, -st.mh));
+
+template <typename T> __device__ __forceinline__ void add_chunk(const uint4 &w, float nmh, Online &st);
+template <> __device__ __forceinline__ void add_chunk<float>(const uint4 &w, float nmh, Online &st) {
+    const float2 sc = make_float2(kLog2e, kLog2e), nm = make_float2(nmh, nmh);
+    st.Sa = fadd2(st.Sa, exp2_pair(make_float2(__uint_as_float(w.x), __uint_as_float(w.y)), sc, nm));
+    st.Sb = fadd2(st.Sb, exp2_pair(make_float2(__uint_as_float(w.z), __uint_as_float(w.w)), sc, nm));
+}
+template <> __device__ __forceinline__ void add_chunk<bf16_t>(const uint4 &w, float nmh, Online &st) {
+    const float2 sc = make_float2(kLog2e, kLog2e), nm = make_float2(nmh, nmh);
+    st.Sa = fadd2(st.Sa, exp2_pair(make_float2(bf16_lo(w.x), bf16_hi(w.x)), sc, nm));
+    st.Sb = fadd2(st.Sb, exp2_pair(make_float2(bf16_lo(w.y), bf16_hi(w.y)), sc, nm));
+    st.Sa = fadd2(st.Sa, exp2_pair(make_float2(bf16_lo(w.z), bf16_hi(w.z)), sc, nm));
+    st.Sb = fadd2(st.Sb, exp2_pair(make_float2(bf16_lo(w.w), bf16_hi(w.w)), sc, nm));
+}
+
+// Adds this thread's chunks (ct, ct + NT, ...) of a stage holding n chunks to its running sum.
+template <typename T>
+__device__ __forceinline__ void add_chunks(uint32_t a0, int n, int ct, int NT, Online &st) {
+    const float nmh = -st.mh;
+    int c = ct;
+    for (; c + 3 * NT < n; c += 4 * NT) {
+        const uint4 w0 = lds128(a0 + (uint32_t)c * 16);
+        const uint4 w1 = lds128(a0 + (uint32_t)(c + NT) * 16);
+        const uint4 w2 = lds128(a0 + (uint32_t)(c + 2 * NT) * 16);
+        const uint4 w3 = lds128(a0 + (uint32_t)(c + 3 * NT) * 16);
+        add_chunk<T>(w0, nmh, st);
+        add_chunk<T>(w1, nmh, st);
+        add_chunk<T>(w2, nmh, st);
+        add_chunk<T>(w3, nmh, st);
+    }
+    for (; c < n; c += NT) {
+        const uint4 w = lds128(a0 + (uint32_t)c * 16);
+        add_chunk<T>(w, nmh, st);
+    }
+}
+
+template <typename T>
+__device__ __forceinline__ void consume_stage(uint32_t a0, int n, int ct, int NT, Online &st) {
+    if (ct >= n) return;
+    if (!(st.m > -INFINITY)) {
+        // no reference yet (start of a row): the largest element of the first chunk
+        const float cm = chunk_max<T>(lds128(a0 + (uint32_t)ct * 16));
+        if (cm > -INFINITY) { st.m = cm; st.mh = cm * kLog2e; }
+    }
+    const Online saved = st;
+    add_chunks<T>(a0, n, ct, NT, st);
+    if (!(st.total() < kSumLimit)) {
+        // an element far above the reference, a NaN or +inf, or only -inf so far: redo the
+        // stage relative to the maximum of this thread's chunks
+        st = saved;
+        float cm = -INFINITY;
+        for (int c = ct; c < n; c += NT) cm = fmaxf(cm, chunk_max<T>(lds128(a0 + (uint32_t)c * 16)));
+        if (cm > st.m) st.raise_to(cm);
+        if (st.m > -INFINITY) add_chunks<T>(a0, n, ct, NT, st);
+    }
 }
 
 // Warp-level merge of the lanes' (m, S) into one pair relative to the warp maximum.
 __device__ __forceinline__ float2 warp_merge(const Online &st) {
-    const float S = (st.S0 + st.S1) + (st.S2 + st.S3);
+    const float S = st.total();
     const float ml = fmaf(st.m, kLog2e, -st.mh);        // exponents carried +ml: take it out
     const float M = warp_max(st.m);
-    // S == 0 covers lanes that saw nothing (their ml is meaningless); a NaN sum still propagates
+    // S == 0 covers lanes that saw nothing (their m is -inf); a NaN sum still propagates
     const float Sw = warp_sum(S == 0.f ? 0.f : S * ex2(fmaf(st.m - M, kLog2e, -ml)));
     return make_float2(M, Sw);
 }
@@ -128,48 +176,48 @@ __global__ void __launch_bounds__(544, 1) verify_rows_tma(const VerifyParams p) 
     if (warp == 0) {
         // =============================== producer ===============================
         const int64_t *offs = cache_off ? off_cache : p.tok_off;
-        int64_t it = 0;             // stages handed out so far
+        int s = 0;                  // stage to fill next, and the phase of its barriers
+        uint32_t ph = 0;
         bool failed = false;
+        const int max_chunks = p.stage_bytes >> 4;
         for (int64_t k0 = 0; !failed; k0 += 32) {
             const int64_t first = (int64_t)blockIdx.x + k0 * gridDim.x;
             if (first >= p.num_items) break;
             const int64_t mine = first + (int64_t)lane * gridDim.x;
+            const int64_t my_row = mine / p.split;
             bool active = mine < p.num_items;
             if (active && p.skip) {
-                const int b = utterance_of_row(offs, p.B, mine / p.split);
+                const int b = utterance_of_row(offs, p.B, my_row);
                 active = !(b >= 0 && p.skip[b]);
             }
             unsigned todo = __ballot_sync(0xffffffffu, active);
             while (todo && !failed) {
                 const int src = __ffs(todo) - 1;
                 todo &= todo - 1;
-                const int64_t item = __shfl_sync(0xffffffffu, mine, src);
-                const int64_t row = item / p.split;
-                const int sp = (int)(item - row * p.split);
+                const int64_t row = __shfl_sync(0xffffffffu, my_row, src);
+                const int sp = (int)(__shfl_sync(0xffffffffu, mine, src) - row * p.split);
                 const uintptr_t g0 = reinterpret_cast<uintptr_t>(p.logits) +
                                      (uintptr_t)(row * p.ld * ES);
                 const uintptr_t g1 = g0 + (uintptr_t)row_bytes;
                 const uintptr_t f0 = g0 & ~(uintptr_t)15;
-                const int64_t row_chunks = (int64_t)((((g1 + 15) & ~(uintptr_t)15) - f0) >> 4);
-                const int64_t cps = (row_chunks + p.split - 1) / p.split;
-                const int64_t sc0 = min(row_chunks, sp * cps), sc1 = min(row_chunks, sc0 + cps);
-                const int64_t span = sc1 - sc0;
-                const int64_t max_chunks = p.stage_bytes >> 4;
-                const int64_t parts = span > 0 ? (span + max_chunks - 1) / max_chunks : 1;
-                const int64_t per_part = span > 0 ? (span + parts - 1) / parts : 0;
+                const int row_chunks = (int)((((g1 + 15) & ~(uintptr_t)15) - f0) >> 4);
+                const int cps = (row_chunks + p.split - 1) / p.split;
+                const int sc0 = min(row_chunks, sp * cps), sc1 = min(row_chunks, sc0 + cps);
+                const int span = sc1 - sc0;
+                const int parts = span > 0 ? (span + max_chunks - 1) / max_chunks : 1;
+                const int per_part = span > 0 ? (span + parts - 1) / parts : 0;
                 const int64_t slot = row * p.partials_per_row + (int64_t)sp * CW;
-                for (int64_t part = 0; part < parts && !failed; ++part, ++it) {
-                    const int s = (int)(it % S);
-                    const uint32_t ph = (uint32_t)((it / S) & 1);
+                const bool head_ragged = f0 != g0, tail_ragged = (g1 & 15) != 0;
+                for (int part = 0; part < parts; ++part) {
                     if (!mbar_wait_bounded(empty0 + s * 8, ph ^ 1u)) { failed = true; break; }
-                    const int64_t pc0 = sc0 + part * per_part;
-                    const int64_t pc1 = min(sc1, pc0 + per_part);
+                    const int pc0 = sc0 + part * per_part;
+                    const int pc1 = min(sc1, pc0 + per_part);
                     // chunks that are only partly inside the row (row start / end not on a
                     // 16-byte boundary) are filled here with plain loads and -inf padding; the
                     // bulk copy takes the fully valid chunks only, so it never leaves the row.
-                    int64_t b0 = pc0, b1 = pc1;
+                    int b0 = pc0, b1 = pc1;
                     unsigned char *dst = stage0_ptr + (size_t)s * p.stage_bytes;
-                    if (pc1 > pc0 && pc0 == 0 && f0 != g0) {
+                    if (head_ragged && pc1 > pc0 && pc0 == 0) {
                         b0 = 1;
                         if (lane < EPC) {
                             const uintptr_t a = f0 + (uintptr_t)lane * ES;
@@ -180,7 +228,7 @@ __global__ void __launch_bounds__(544, 1) verify_rows_tma(const VerifyParams p) 
                                 ok ? *reinterpret_cast<const uint16_t *>(a) : (uint16_t)0xff80u;
                         }
                     }
-                    if (pc1 > pc0 && pc1 == row_chunks && (g1 & 15) != 0 &&
+                    if (tail_ragged && pc1 > pc0 && pc1 == row_chunks &&
                         !(b0 == 1 && row_chunks == 1)) {
                         b1 = pc1 - 1;
                         if (lane < EPC) {
@@ -195,28 +243,27 @@ __global__ void __launch_bounds__(544, 1) verify_rows_tma(const VerifyParams p) 
                     }
                     __syncwarp();
                     if (lane == 0) {
-                        desc[s].nchunks = (int32_t)(pc1 - pc0);
+                        desc[s].nchunks = pc1 - pc0;
                         desc[s].flags = (part == parts - 1) ? kFlagLast : 0u;
                         desc[s].slot = slot;
                         const uint32_t bar = full0 + s * 8;
                         if (b1 > b0) {
-                            const uint32_t bytes = (uint32_t)((b1 - b0) << 4);
+                            const uint32_t bytes = (uint32_t)(b1 - b0) << 4;
                             fence_proxy_async();
                             mbar_arrive_expect_tx(bar, bytes);
-                            bulk_g2s(stage0 + (uint32_t)s * p.stage_bytes + (uint32_t)((b0 - pc0) << 4),
-                                     reinterpret_cast<const void *>(f0 + (uintptr_t)(b0 << 4)),
+                            bulk_g2s(stage0 + (uint32_t)s * p.stage_bytes + ((uint32_t)(b0 - pc0) << 4),
+                                     reinterpret_cast<const void *>(f0 + ((uintptr_t)b0 << 4)),
                                      bytes, bar);
                         } else {
                             mbar_arrive(bar);
                         }
                     }
                     __syncwarp();
+                    if (++s == S) { s = 0; ph ^= 1u; }
                 }
             }
         }
         if (!failed) {
-            const int s = (int)(it % S);
-            const uint32_t ph = (uint32_t)((it / S) & 1);
             if (mbar_wait_bounded(empty0 + s * 8, ph ^ 1u)) {
                 if (lane == 0) {
                     desc[s].nchunks = 0; desc[s].flags = kFlagEnd; desc[s].slot = 0;
@@ -237,30 +284,16 @@ __global__ void __launch_bounds__(544, 1) verify_rows_tma(const VerifyParams p) 
         Online st;
         st.reset();
         bool failed = false;
-        for (int64_t it = 0;; ++it) {
-            const int s = (int)(it % S);
-            const uint32_t ph = (uint32_t)((it / S) & 1);
+        int s = 0;
+        uint32_t ph = 0;
+        for (;;) {
             if (!mbar_wait_bounded(full0 + s * 8, ph)) { failed = true; break; }
             const int n = desc[s].nchunks;
             const uint32_t flags = desc[s].flags;
-            const int64_t slot = desc[s].slot;
             if (flags & kFlagEnd) break;
-            const uint32_t a0 = stage0 + (uint32_t)s * p.stage_bytes;
-            int c = ct;
-            for (; c + 3 * NT < n; c += 4 * NT) {
-                const uint4 w0 = lds128(a0 + (uint32_t)c * 16);
-                const uint4 w1 = lds128(a0 + (uint32_t)(c + NT) * 16);
-                const uint4 w2 = lds128(a0 + (uint32_t)(c + 2 * NT) * 16);
-                const uint4 w3 = lds128(a0 + (uint32_t)(c + 3 * NT) * 16);
-                consume_chunk<T>(w0, st);
-                consume_chunk<T>(w1, st);
-                consume_chunk<T>(w2, st);
-                consume_chunk<T>(w3, st);
-            }
-            for (; c < n; c += NT) {
-                const uint4 w = lds128(a0 + (uint32_t)c * 16);
-                consume_chunk<T>(w, st);
-            }
+            consume_stage<T>(stage0 + (uint32_t)s * p.stage_bytes, n, ct, NT, st);
+            int64_t slot = 0;
+            if (flags & kFlagLast) slot = desc[s].slot;
             __syncwarp();
             if (lane == 0) mbar_arrive(empty0 + s * 8);
             if (flags & kFlagLast) {
@@ -268,6 +301,7 @@ __global__ void __launch_bounds__(544, 1) verify_rows_tma(const VerifyParams p) 
                 if (lane == 0) p.partials[slot + cw] = r;
                 st.reset();
             }
+            if (++s == S) { s = 0; ph ^= 1u; }
         }
         if (failed) {
             if (lane == 0) atomicExch(p.err_word, p.epoch);
@@ -389,10 +423,33 @@ int plan_verify(int B, int64_t M, int V, ssd_dtype dtype, const ssd_launch_opts 
     const int sms = device_sm_count();
     pl.ctas = (o && o->ctas > 0) ? o->ctas : sms;
     const int64_t row_bytes = (int64_t)V * es;
+    // column spans per row: enough items for a few balanced waves when there are few rows
+    int split = 1;
+    if (o && o->split > 0) {
+        split = o->split;
+    } else if (M > 0 && M < 8ll * pl.ctas) {
+        const int64_t want = (8ll * pl.ctas + M - 1) / M;
+        const int64_t most = row_bytes / 16384 > 1 ? row_bytes / 16384 : 1;  // spans >= 16 KB
+        split = (int)(want < most ? want : most);
+    }
+    if (split < 1) split = 1;
+    if (split > 64) split = 64;
+    pl.split = split;
     if (pl.kernel == 2) {
-        pl.warps = (o && o->warps > 0) ? o->warps : 8;
+        pl.warps = (o && o->warps > 0) ? o->warps : 16;
         if (pl.warps > 16) return SSD_ERR_ARG;
-        pl.stage_bytes = (o && o->stage_bytes > 0) ? o->stage_bytes : 32768;
+        if (o && o->stage_bytes > 0) {
+            pl.stage_bytes = o->stage_bytes;
+        } else {
+            // a span is cut into equal parts of at most 64 KB, one part per stage: few, large
+            // stages keep the per-stage handshake off the critical path
+            const int64_t span = (row_bytes + split - 1) / split + 32;
+            const int64_t parts = (span + 65535) / 65536;
+            int64_t sb = ((span + parts - 1) / parts + 16 + 127) & ~127ll;
+            if (sb < 4096) sb = 4096;
+            if (sb > 65536) sb = 65536;
+            pl.stage_bytes = (int)sb;
+        }
         if (pl.stage_bytes < 1024 || pl.stage_bytes > 65536 || (pl.stage_bytes & 127))
             return SSD_ERR_ARG;
         const int off_cache = (B + 1 <= kOffCacheMax) ? (B + 1) * 8 : 0;
@@ -407,18 +464,6 @@ int plan_verify(int B, int64_t M, int V, ssd_dtype dtype, const ssd_launch_opts 
         pl.warps = 8;
         pl.stages = 0; pl.stage_bytes = 0; pl.smem_bytes = 0;
     }
-    // column spans per row: enough items for a few balanced waves when there are few rows
-    int split = 1;
-    if (o && o->split > 0) {
-        split = o->split;
-    } else if (M > 0 && M < 8ll * pl.ctas) {
-        const int64_t want = (8ll * pl.ctas + M - 1) / M;
-        const int64_t most = row_bytes / 16384 > 1 ? row_bytes / 16384 : 1;  // spans >= 16 KB
-        split = (int)(want < most ? want : most);
-    }
-    if (split < 1) split = 1;
-    if (split > 64) split = 64;
-    pl.split = split;
     pl.partials = split * pl.warps;
     pl.workspace_bytes = 256 + (size_t)M * pl.partials * sizeof(float2);
     *plan = pl;

@@ -112,7 +112,7 @@ def test_workspace_queries(lib):
     big = ssd.ssd_verify_workspace_bytes(32, 6400, 49152, ssd.BF16)
     assert small >= 256 + 250 * 8 * 8 and big >= 256 + 6400 * 8 * 8
     o = ssd.LaunchOpts()
-    o.split = 4
+    o.split, o.warps = 4, 8
     assert ssd.ssd_verify_workspace_bytes(32, 6400, 49152, ssd.BF16, o) == 256 + 6400 * 4 * 8 * 8
 
 
