@@ -137,6 +137,29 @@ __device__ __forceinline__ uint32_t bf16x2_max(uint32_t a, uint32_t b) {
     return d;
 }
 
+// the same, but a NaN operand wins (so that a NaN logit is not swallowed by a clamp)
+__device__ __forceinline__ uint32_t bf16x2_max_nan(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ float fmax_nan(float a, float b) {
+    float d;
+    asm("max.NaN.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+    return d;
+}
+
+// (lo, hi) halves of a packed bf16 pair, each plus c, in fp32: the mixed-precision add of
+// sm_100 reads the 16-bit halves directly, so no unpacking instruction is needed.
+__device__ __forceinline__ float2 bf16x2_add_f32(uint32_t w, float c) {
+    float2 d;
+    asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\t"
+        "add.rn.f32.bf16 %0, lo, %3;\n\tadd.rn.f32.bf16 %1, hi, %3;\n\t}"
+        : "=f"(d.x), "=f"(d.y)
+        : "r"(w), "f"(c));
+    return d;
+}
+
 // order-preserving map float -> int32 (for integer warp reductions of float maxima)
 __device__ __forceinline__ int32_t float_key(float f) {
     int32_t b = __float_as_int(f);

@@ -36,105 +36,277 @@ struct CtcParams {
     float *frame_logprob;
 };
 
-// Statistics of one row held by one warp.
-struct RowStats {
-    float lse, entropy;
+// Replaces the elements of a 16-byte chunk outside [e_lo, e_hi) (they belong to a neighbouring
+// row, to the padding between rows, or were never written) by -inf, or, with kFinite, by a
+// finite value near -1e30 whose exponential is 0 and whose product with that 0 is not NaN.
+template <typename T, bool kFinite>
+__device__ __forceinline__ void mask_chunk(uint4 &w, int e_lo, int e_hi);
+template <bool kFinite> __device__ __forceinline__ void mask_f32(uint4 &w, int e_lo, int e_hi) {
+    const uint32_t fill = kFinite ? 0xf149f2cau : 0xff800000u;
+    if (0 < e_lo || 0 >= e_hi) w.x = fill;
+    if (1 < e_lo || 1 >= e_hi) w.y = fill;
+    if (2 < e_lo || 2 >= e_hi) w.z = fill;
+    if (3 < e_lo || 3 >= e_hi) w.w = fill;
+}
+template <bool kFinite>
+__device__ __forceinline__ uint32_t mask_pair(uint32_t v, int j, int e_lo, int e_hi) {
+    const uint32_t fill = kFinite ? 0xf149u : 0xff80u;
+    if (j < e_lo || j >= e_hi) v = (v & 0xffff0000u) | fill;
+    if (j + 1 < e_lo || j + 1 >= e_hi) v = (v & 0x0000ffffu) | (fill << 16);
+    return v;
+}
+template <bool kFinite> __device__ __forceinline__ void mask_bf16(uint4 &w, int e_lo, int e_hi) {
+    w.x = mask_pair<kFinite>(w.x, 0, e_lo, e_hi);
+    w.y = mask_pair<kFinite>(w.y, 2, e_lo, e_hi);
+    w.z = mask_pair<kFinite>(w.z, 4, e_lo, e_hi);
+    w.w = mask_pair<kFinite>(w.w, 6, e_lo, e_hi);
+}
+template <> __device__ __forceinline__ void mask_chunk<float, false>(uint4 &w, int a, int b) { mask_f32<false>(w, a, b); }
+template <> __device__ __forceinline__ void mask_chunk<float, true>(uint4 &w, int a, int b) { mask_f32<true>(w, a, b); }
+template <> __device__ __forceinline__ void mask_chunk<bf16_t, false>(uint4 &w, int a, int b) { mask_bf16<false>(w, a, b); }
+template <> __device__ __forceinline__ void mask_chunk<bf16_t, true>(uint4 &w, int a, int b) { mask_bf16<true>(w, a, b); }
+
+// S += 2^t, A += t * 2^t for the elements of one chunk, t = x*log2e - mh.  Elements are first
+// clamped from below so that a masked (-inf) logit gives t*2^t = 0 instead of NaN.
+template <typename T>
+__device__ __forceinline__ void entropy_chunk(const uint4 &w, float nmh, float2 &Sa, float2 &Sb,
+                                              float2 &Aa, float2 &Ab);
+__device__ __forceinline__ void entropy_pair(float2 x, float nmh, float2 &S, float2 &A) {
+    const float2 t = ffma2(x, make_float2(kLog2e, kLog2e), make_float2(nmh, nmh));
+    const float2 e = make_float2(ex2(t.x), ex2(t.y));
+    S = fadd2(S, e);
+    A = ffma2(t, e, A);
+}
+template <>
+__device__ __forceinline__ void entropy_chunk<float>(const uint4 &w, float nmh, float2 &Sa,
+                                                     float2 &Sb, float2 &Aa, float2 &Ab) {
+    const float lo = -1.0e30f;
+    entropy_pair(make_float2(fmax_nan(__uint_as_float(w.x), lo), fmax_nan(__uint_as_float(w.y), lo)),
+                 nmh, Sa, Aa);
+    entropy_pair(make_float2(fmax_nan(__uint_as_float(w.z), lo), fmax_nan(__uint_as_float(w.w), lo)),
+                 nmh, Sb, Ab);
+}
+template <>
+__device__ __forceinline__ void entropy_chunk<bf16_t>(const uint4 &w, float nmh, float2 &Sa,
+                                                      float2 &Sb, float2 &Aa, float2 &Ab) {
+    const uint32_t lo = 0xf149f149u;      // bf16 pair of -1.0e30 (rounded)
+    const uint32_t x = bf16x2_max_nan(w.x, lo), y = bf16x2_max_nan(w.y, lo);
+    const uint32_t z = bf16x2_max_nan(w.z, lo), u = bf16x2_max_nan(w.w, lo);
+    entropy_pair(make_float2(bf16_lo(x), bf16_hi(x)), nmh, Sa, Aa);
+    entropy_pair(make_float2(bf16_lo(y), bf16_hi(y)), nmh, Sb, Ab);
+    entropy_pair(make_float2(bf16_lo(z), bf16_hi(z)), nmh, Sa, Aa);
+    entropy_pair(make_float2(bf16_lo(u), bf16_hi(u)), nmh, Sb, Ab);
+}
+
+template <int G> __device__ __forceinline__ float group_max(float v) {
+#pragma unroll
+    for (int o = G / 2; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+template <int G> __device__ __forceinline__ int group_min(int v) {
+#pragma unroll
+    for (int o = G / 2; o > 0; o >>= 1) v = min(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+template <int G> __device__ __forceinline__ float group_sum(float v) {
+#pragma unroll
+    for (int o = G / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+struct RowOut {
+    float lse, H;
     int arg;
 };
 
-template <typename T>
-__device__ __forceinline__ void accumulate(float x, float mh, float &S, float &A) {
-    float t2 = fmaf(x, kLog2e, -mh);
-    float e = ex2(t2);
-    S += e;
-    A = fmaf(fmaxf(t2, -200.f), e, A);   // the clamp turns (-inf)*0 into 0
-}
+// Geometry of one row inside a stage: the 16-byte chunks [cf, cl] it touches and which
+// elements of the first and last chunk are its own.
+struct RowSpan {
+    int cf, cl, e_lo, e_hi;
+};
 
-// Reduces one row that lies in shared memory at byte address `row_addr` (element aligned).
-// Exact two-pass softmax: pass 1 finds the maximum and where it first occurs, pass 2 sums
-// e = 2^((x-m)*log2e) and (x-m)*log2e*e.  With mh = fl(m*log2e) and ml = m*log2e - mh (exact,
-// by fma) every exponent carries the same +ml, which cancels in the entropy and is removed
-// from the log-sum-exp at the end.
-template <typename T>
-__device__ __forceinline__ RowStats reduce_row_smem(uint32_t stage_addr, uint32_t row_off,
-                                                    int V, int lane) {
-    constexpr int ES = Elem<T>::kBytes, EPC = Elem<T>::kPerChunk;
-    const int e0 = row_off / ES;                 // element offset of the row inside the stage
-    int c0 = (e0 + EPC - 1) / EPC;               // first full 16-byte chunk
-    int c1 = (e0 + V) / EPC;                     // one past the last full chunk
-    int nhead, ntail;
-    if (c1 > c0) { nhead = c0 * EPC - e0; ntail = e0 + V - c1 * EPC; }
-    else { c0 = c1 = 0; nhead = V; ntail = 0; }
-    const int tail0 = c1 * EPC - e0;             // row-relative index of the first tail element
-
-    // ---- pass 1: maximum and its first position among this lane's elements ----
+// Exact two-pass softmax of one row by the G lanes of a group (all 32 lanes call it).  Pass 1
+// finds the maximum m and where it first occurs, pass 2 sums e = 2^((x-m)*log2e) and
+// (x-m)*log2e*e with masked logits clamped.  With mh = fl(m*log2e) and ml = m*log2e - mh
+// (exact, by fma) every exponent carries the same +ml, which cancels in the entropy and is
+// removed from the log-sum-exp at the end.  This is the path for rows the fused pass below
+// cannot take (masked -inf logits, NaN, +inf, a dynamic range beyond fp32's exponent).
+template <typename T, int G>
+__device__ __noinline__ RowOut reduce_row_exact(uint32_t stage_addr, RowSpan r, int sub) {
+    constexpr int EPC = Elem<T>::kPerChunk;
+    const int cf = r.cf, cl = r.cl, e_lo = r.e_lo, e_hi = r.e_hi;
     float vmax = -INFINITY;
-    int vidx = INT_MAX;
-    bool vchunk = false;
-    for (int i = lane; i < nhead; i += 32) {
-        float x = Elem<T>::load_shared(stage_addr + (e0 + i) * ES);
-        if (x > vmax) { vmax = x; vidx = i; }
+    int vc = -1;
+    for (int c = cf + sub; c <= cl; c += G) {
+        uint4 w = lds128(stage_addr + (uint32_t)c * 16);
+        if (c == cf || c == cl) mask_chunk<T, false>(w, c == cf ? e_lo : 0, c == cl ? e_hi : EPC);
+        const float cm = chunk_max<T>(w);
+        if (cm > vmax) { vmax = cm; vc = c; }
     }
-#pragma unroll 4
-    for (int c = c0 + lane; c < c1; c += 32) {
-        uint4 w = lds128(stage_addr + c * 16);
-        float cm = chunk_max<T>(w);
-        if (cm > vmax) { vmax = cm; vidx = c * EPC - e0; vchunk = true; }
-    }
-    for (int i = lane; i < ntail; i += 32) {
-        float x = Elem<T>::load_shared(stage_addr + (e0 + tail0 + i) * ES);
-        if (x > vmax) { vmax = x; vidx = tail0 + i; vchunk = false; }
-    }
-    const float m = warp_max(vmax);
+    const float m = group_max<G>(vmax);
     int cand = INT_MAX;
-    if (vmax == m && vidx != INT_MAX) {
-        cand = vidx;
-        if (vchunk) {
-            uint4 w = lds128(stage_addr + (e0 + vidx) * ES);
-            float x[EPC];
-            chunk_unpack<T>(w, x);
-            int j = EPC - 1;
-#pragma unroll
-            for (int k = EPC - 2; k >= 0; --k) if (x[k] == m) j = k;
-            cand = vidx + j;
-        }
-    }
-    int arg = __reduce_min_sync(0xffffffffu, cand);
-    if (arg == INT_MAX) arg = 0;
-
-    // ---- pass 2: sums ----
-    const float mh = m * kLog2e;
-    const float ml = fmaf(m, kLog2e, -mh);
-    float S0 = 0.f, S1 = 0.f, A0 = 0.f, A1 = 0.f;
-    for (int i = lane; i < nhead; i += 32)
-        accumulate<T>(Elem<T>::load_shared(stage_addr + (e0 + i) * ES), mh, S0, A0);
-    for (int i = lane; i < ntail; i += 32)
-        accumulate<T>(Elem<T>::load_shared(stage_addr + (e0 + tail0 + i) * ES), mh, S1, A1);
-#pragma unroll 4
-    for (int c = c0 + lane; c < c1; c += 32) {
-        uint4 w = lds128(stage_addr + c * 16);
+    if (vc >= 0 && vmax == m) {
+        uint4 w = lds128(stage_addr + (uint32_t)vc * 16);
+        if (vc == cf || vc == cl) mask_chunk<T, false>(w, vc == cf ? e_lo : 0, vc == cl ? e_hi : EPC);
         float x[EPC];
         chunk_unpack<T>(w, x);
+        int j = EPC - 1;
 #pragma unroll
-        for (int k = 0; k < EPC; k += 2) {
-            accumulate<T>(x[k], mh, S0, A0);
-            accumulate<T>(x[k + 1], mh, S1, A1);
-        }
+        for (int k = EPC - 2; k >= 0; --k) if (x[k] == m) j = k;
+        cand = (vc - cf) * EPC + j - e_lo;
     }
-    const float S = warp_sum(S0 + S1);
-    const float A2 = warp_sum(A0 + A1);
-    RowStats r;
+    RowOut out;
+    out.arg = group_min<G>(cand);
+    if (out.arg == INT_MAX) out.arg = 0;
+    const float mh = m * kLog2e;
+    const float ml = fmaf(m, kLog2e, -mh);
+    float2 Sa = make_float2(0.f, 0.f), Sb = Sa, Aa = Sa, Ab = Sa;
+    for (int c = cf + sub; c <= cl; c += G) {
+        uint4 w = lds128(stage_addr + (uint32_t)c * 16);
+        if (c == cf || c == cl) mask_chunk<T, false>(w, c == cf ? e_lo : 0, c == cl ? e_hi : EPC);
+        entropy_chunk<T>(w, -mh, Sa, Sb, Aa, Ab);
+    }
+    const float S = group_sum<G>((Sa.x + Sa.y) + (Sb.x + Sb.y));
+    const float A2 = group_sum<G>((Aa.x + Aa.y) + (Ab.x + Ab.y));
     const float lnS = logf(S);
-    r.lse = m + (lnS - ml * kLn2);
-    r.entropy = fmaxf(lnS - kLn2 * (A2 / S), 0.f);
+    out.lse = m + (lnS - ml * kLn2);
+    out.H = fmaxf(lnS - kLn2 * (A2 / S), 0.f);
     if (!(S > 0.5f) || !(S < INFINITY) || !(fabsf(m) < INFINITY))
-        r.entropy = __int_as_float(0x7fc00000);   // NaN / +inf / all -inf: flagged downstream
-    r.arg = arg;
-    return r;
+        out.H = __int_as_float(0x7fc00000);       // NaN / +inf / all -inf: flagged downstream
+    return out;
 }
 
+// One chunk of the fused pass: running maximum (with the chunk it was first met in) and the
+// sums S += 2^t, A += t*2^t with t = x*log2e - rh for a per-lane reference rh (in log2 units).
 template <typename T>
-__global__ void __launch_bounds__(512, 1) ctc_rows_tma(const CtcParams p) {
+__device__ __forceinline__ void fused_chunk(const uint4 &w, int c, float nrh, float &vmax, int &vc,
+                                            float2 &Sa, float2 &Sb, float2 &Aa, float2 &Ab);
+template <>
+__device__ __forceinline__ void fused_chunk<float>(const uint4 &w, int c, float nrh, float &vmax,
+                                                   int &vc, float2 &Sa, float2 &Sb, float2 &Aa,
+                                                   float2 &Ab) {
+    const float cm = chunk_max<float>(w);
+    if (cm > vmax) { vmax = cm; vc = c; }
+    entropy_pair(make_float2(__uint_as_float(w.x), __uint_as_float(w.y)), nrh, Sa, Aa);
+    entropy_pair(make_float2(__uint_as_float(w.z), __uint_as_float(w.w)), nrh, Sb, Ab);
+}
+template <>
+__device__ __forceinline__ void fused_chunk<bf16_t>(const uint4 &w, int c, float nrh, float &vmax,
+                                                    int &vc, float2 &Sa, float2 &Sb, float2 &Aa,
+                                                    float2 &Ab) {
+    const float cm = chunk_max<bf16_t>(w);
+    if (cm > vmax) { vmax = cm; vc = c; }
+    entropy_pair(make_float2(bf16_lo(w.x), bf16_hi(w.x)), nrh, Sa, Aa);
+    entropy_pair(make_float2(bf16_lo(w.y), bf16_hi(w.y)), nrh, Sb, Ab);
+    entropy_pair(make_float2(bf16_lo(w.z), bf16_hi(w.z)), nrh, Sa, Aa);
+    entropy_pair(make_float2(bf16_lo(w.w), bf16_hi(w.w)), nrh, Sb, Ab);
+}
+
+// Frame statistics of the rows of one tile that lies in shared memory.  G lanes share a row
+// and a warp works on 32/G rows at a time.  A row is walked in the 16-byte chunks of the stage
+// (whose alignment is that of global memory); its first and last chunk may also hold foreign
+// elements, which are masked.
+//
+// Fused single pass: a lane takes the largest element of its first chunk as reference (rh =
+// fl(ref*log2e), in log2 units) and, for every chunk, updates its running maximum and adds 2^t
+// and t*2^t, t = x*log2e - rh (one fma).  fp32 keeps full relative precision whatever the
+// reference, so the sums only have to stay in range; at the end the lanes' sums are re-based
+// to mh = fl(m*log2e) of the row maximum m (S' = S*2^d, A' = (A + d*S)*2^d with d = rh - mh,
+// an exact difference) and added; ml = m*log2e - mh (exact, by fma) is taken out of the
+// log-sum-exp and cancels in the entropy.  One exponential per logit, and
+// the comparisons overlap with the exponentials.  A group whose sums left the range or turned
+// NaN (a logit far above the reference, masked -inf logits, NaN, +inf) is redone by the exact
+// two-pass routine above.
+template <typename T, int G>
+__device__ __forceinline__ void reduce_tile(const CtcParams &p, uint32_t stage_addr, uint32_t head,
+                                            int64_t r0, int nrows, int lane) {
+    constexpr int ES = Elem<T>::kBytes, EPC = Elem<T>::kPerChunk, RPW = 32 / G;
+    const int sub = lane % G, grp = lane / G;
+    const uint32_t pitch = (uint32_t)(p.ld * ES), row_bytes = (uint32_t)p.V * ES;
+    for (int g0 = 0; g0 < nrows; g0 += RPW) {
+        const int i = g0 + grp;
+        const bool valid = i < nrows;
+        const uint32_t off = head + (uint32_t)(valid ? i : 0) * pitch;
+        RowSpan r;
+        r.cf = (int)(off >> 4);
+        r.cl = valid ? (int)((off + row_bytes - 1) >> 4) : r.cf - 1;
+        r.e_lo = (int)(off & 15) / ES;
+        r.e_hi = (int)((off + row_bytes - 1) & 15) / ES + 1;
+        const int cf = r.cf, cl = r.cl;
+
+        float vmax = -INFINITY, ref = 0.f;
+        int vc = -1;
+        float2 Sa = make_float2(0.f, 0.f), Sb = Sa, Aa = Sa, Ab = Sa;
+        int c = cf + sub;
+        if (c <= cl) {
+            // first chunk of this lane (an edge chunk for some lanes): fixes the reference
+            uint4 w = lds128(stage_addr + (uint32_t)c * 16);
+            if (c == cf || c == cl) mask_chunk<T, true>(w, c == cf ? r.e_lo : 0, c == cl ? r.e_hi : EPC);
+            const float cm = chunk_max<T>(w);
+            if (cm > -INFINITY) ref = cm * kLog2e;
+            fused_chunk<T>(w, c, -ref, vmax, vc, Sa, Sb, Aa, Ab);
+            c += G;
+#pragma unroll 2
+            for (; c < cl; c += G) {           // interior chunks: no masks
+                const uint4 wi = lds128(stage_addr + (uint32_t)c * 16);
+                fused_chunk<T>(wi, c, -ref, vmax, vc, Sa, Sb, Aa, Ab);
+            }
+            if (c == cl) {                      // the row's last chunk
+                uint4 wl = lds128(stage_addr + (uint32_t)c * 16);
+                mask_chunk<T, true>(wl, 0, r.e_hi);
+                fused_chunk<T>(wl, c, -ref, vmax, vc, Sa, Sb, Aa, Ab);
+            }
+        }
+        const float Sl = (Sa.x + Sa.y) + (Sb.x + Sb.y), Al = (Aa.x + Aa.y) + (Ab.x + Ab.y);
+        // out of range, NaN, or a lane that saw nothing above the mask fill value
+        const bool bad = !(Sl < 1.0e30f) || Al != Al || (vc >= 0 && !(vmax > -1.0e29f));
+        RowOut out;
+        if (__any_sync(0xffffffffu, bad)) {
+            out = reduce_row_exact<T, G>(stage_addr, r, sub);
+        } else {
+            const float m = group_max<G>(vmax);
+            int cand = INT_MAX;
+            if (vc >= 0 && vmax == m) {
+                uint4 w = lds128(stage_addr + (uint32_t)vc * 16);
+                if (vc == cf || vc == cl)
+                    mask_chunk<T, true>(w, vc == cf ? r.e_lo : 0, vc == cl ? r.e_hi : EPC);
+                float x[EPC];
+                chunk_unpack<T>(w, x);
+                int j = EPC - 1;
+#pragma unroll
+                for (int k = EPC - 2; k >= 0; --k) if (x[k] == m) j = k;
+                cand = (vc - cf) * EPC + j - r.e_lo;
+            }
+            out.arg = group_min<G>(cand);
+            if (out.arg == INT_MAX) out.arg = 0;
+            const float mh = m * kLog2e;
+            const float ml = fmaf(m, kLog2e, -mh);
+            const float d = ref - mh;                    // <= 0; lanes without chunks have S = 0
+            const float sc = ex2(d);
+            const float S = group_sum<G>(Sl * sc);
+            const float A2 = group_sum<G>(fmaf(d, Sl, Al) * sc);
+            // fast logarithm and division: absolute error near 1e-6, far inside the tolerance
+            const float lnS = __logf(S);
+            out.lse = m + (lnS - ml * kLn2);
+            out.H = fmaxf(lnS - kLn2 * __fdividef(A2, S), 0.f);
+            if (!(S > 0.5f) || !(S < INFINITY) || !(fabsf(m) < INFINITY))
+                out.H = __int_as_float(0x7fc00000);
+        }
+        if (valid && sub == 0) {
+            p.frame_entropy[r0 + i] = out.H;
+            p.frame_argmax[r0 + i] = out.arg;
+            if (p.frame_lse) p.frame_lse[r0 + i] = out.lse;
+        }
+        if (p.frame_logprob && valid) {
+            float *o = p.frame_logprob + (r0 + i) * p.ld;
+            for (int a = sub; a < p.V; a += G)
+                o[a] = Elem<T>::load_shared(stage_addr + off + a * ES) - out.lse;
+        }
+    }
+}
+
+template <typename T, int G>
+__global__ void __launch_bounds__(768, 1) ctc_rows_tma(const CtcParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     constexpr int ES = Elem<T>::kBytes;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -160,13 +332,26 @@ __global__ void __launch_bounds__(512, 1) ctc_rows_tma(const CtcParams p) {
 
     // Brings tile k of this warp into stage s.  The tile's rows are one contiguous byte range
     // (padding between rows included); the 16-byte-aligned superset of the range is fetched with
-    // one bulk copy where that superset stays inside the matrix, so that interior tiles need no
-    // scalar fix-up; bytes of neighbouring rows that come along are never looked at.
+    // one bulk copy.  Only for the first and the last tile of the matrix may that superset leave
+    // the matrix: there the bulk copy is shortened and the few elements outside it are fetched
+    // with plain loads.  Bytes of neighbouring rows that come along are never looked at.
+    const int64_t tile_bytes = (int64_t)(R - 1) * row_pitch + (int64_t)p.V * ES;
     auto issue = [&](int64_t k, int s) {
         const int64_t tile = gw + k * GW;
-        const int64_t r0 = tile * R;
-        const int nrows = (int)min((int64_t)R, p.N - r0);
-        const uintptr_t gstart = base + (uintptr_t)(r0 * row_pitch);
+        const uintptr_t gstart = base + (uintptr_t)(tile * R * row_pitch);
+        const uint32_t bar = bar0 + s * 8;
+        if (tile != 0 && tile != p.num_tiles - 1) {
+            if (lane == 0) {
+                const uintptr_t f0 = gstart & ~(uintptr_t)15;
+                const uint32_t bytes = (uint32_t)(((gstart + tile_bytes + 15) & ~(uintptr_t)15) - f0);
+                fence_proxy_async();
+                mbar_arrive_expect_tx(bar, bytes);
+                bulk_g2s(stage0 + (uint32_t)s * p.stage_stride, reinterpret_cast<const void *>(f0),
+                         bytes, bar);
+            }
+            return;
+        }
+        const int nrows = (int)min((int64_t)R, p.N - tile * R);
         const uintptr_t gend = gstart + (uintptr_t)((nrows - 1) * row_pitch + (int64_t)p.V * ES);
         const uintptr_t f0 = gstart & ~(uintptr_t)15;
         const uintptr_t c1 = (gend + 15) & ~(uintptr_t)15;
@@ -175,7 +360,6 @@ __global__ void __launch_bounds__(512, 1) ctc_rows_tma(const CtcParams p) {
         const bool has_bulk = bulk_hi > bulk_lo;
         unsigned char *dst = stage0_ptr + (size_t)s * p.stage_stride;
         if (!has_bulk || bulk_lo > gstart || bulk_hi < gend) {
-            // first / last tile of the matrix only: elements outside the bulk range by plain loads
             const uintptr_t h_end = has_bulk ? min(bulk_lo, gend) : gend;
             for (uintptr_t a = gstart + (uintptr_t)lane * ES; a < h_end; a += 32 * ES) {
                 if (ES == 4) *reinterpret_cast<uint32_t *>(dst + (a - f0)) =
@@ -195,7 +379,6 @@ __global__ void __launch_bounds__(512, 1) ctc_rows_tma(const CtcParams p) {
             __syncwarp();
         }
         if (lane == 0) {
-            const uint32_t bar = bar0 + s * 8;
             if (has_bulk) {
                 const uint32_t bytes = (uint32_t)(bulk_hi - bulk_lo);
                 fence_proxy_async();
@@ -212,46 +395,29 @@ __global__ void __launch_bounds__(512, 1) ctc_rows_tma(const CtcParams p) {
     for (int k = 0; k < prologue; ++k) issue(k, k);
 
     bool failed = false;
-    for (int64_t k = 0; k < my_tiles; ++k) {
-        const int s = (int)(k % S);
-        const uint32_t parity = (uint32_t)((k / S) & 1);
+    int s = 0;
+    uint32_t parity = 0;
+    int64_t k = 0;
+    for (; k < my_tiles; ++k) {
         if (!mbar_wait_bounded(bar0 + s * 8, parity)) { failed = true; break; }
-        const int64_t tile = gw + k * GW;
-        const int64_t r0 = tile * R;
+        const int64_t r0 = (gw + k * GW) * R;
         const int nrows = (int)min((int64_t)R, p.N - r0);
-        const uintptr_t gstart = base + (uintptr_t)(r0 * row_pitch);
-        const uint32_t head = (uint32_t)(gstart & 15);
-        const uint32_t stage_addr = stage0 + (uint32_t)s * p.stage_stride;
-        float myH = 0.f, myL = 0.f;
-        int myA = 0;
-        for (int i = 0; i < nrows; ++i) {
-            const uint32_t row_off = head + (uint32_t)(i * row_pitch);
-            RowStats rs = reduce_row_smem<T>(stage_addr, row_off, p.V, lane);
-            if (lane == i) { myH = rs.entropy; myL = rs.lse; myA = rs.arg; }
-            if (p.frame_logprob) {
-                float *out = p.frame_logprob + (r0 + i) * p.ld;
-                for (int a = lane; a < p.V; a += 32)
-                    out[a] = Elem<T>::load_shared(stage_addr + row_off + a * ES) - rs.lse;
-            }
-        }
-        if (lane < nrows) {
-            p.frame_entropy[r0 + lane] = myH;
-            p.frame_argmax[r0 + lane] = myA;
-            if (p.frame_lse) p.frame_lse[r0 + lane] = myL;
-        }
+        const uint32_t head = (uint32_t)((base + (uintptr_t)(r0 * row_pitch)) & 15);
+        reduce_tile<T, G>(p, stage0 + (uint32_t)s * p.stage_stride, head, r0, nrows, lane);
         __syncwarp();
         if (k + S < my_tiles) issue(k + S, s);
+        if (++s == S) { s = 0; parity ^= 1u; }
     }
     if (failed) {
         // A wait ran out: poison every frame this warp still owed so that the per-utterance
         // kernel reports SSD_UTT_INTERNAL, then let copies that may be in flight land.
-        for (int64_t k = 0; k < my_tiles; ++k) {
+        for (; k < my_tiles; ++k) {
             const int64_t r0 = (gw + k * GW) * R;
             const int nrows = (int)min((int64_t)R, p.N - r0);
-            if (lane < nrows) {
-                p.frame_entropy[r0 + lane] = __uint_as_float(kNanInternal);
-                p.frame_argmax[r0 + lane] = 0;
-                if (p.frame_lse) p.frame_lse[r0 + lane] = __uint_as_float(kNanInternal);
+            for (int i = lane; i < nrows; i += 32) {
+                p.frame_entropy[r0 + i] = __uint_as_float(kNanInternal);
+                p.frame_argmax[r0 + i] = 0;
+                if (p.frame_lse) p.frame_lse[r0 + i] = __uint_as_float(kNanInternal);
             }
         }
         drain_after_error();
@@ -471,34 +637,42 @@ int launch_ctc_rows(const void *logits, ssd_dtype dtype, int V, int64_t ld, int6
     p.frame_logprob = frame_logprob;
 
     // ---- choose the kernel and its shape ----
+    // G lanes share a row (so that a lane walks about 8..18 chunks of 16 bytes), a warp works
+    // on 32/G rows at a time, and a tile is a whole number of such row groups of about 8 KB.
     int kernel = o ? o->kernel : 0;
     const int64_t row_pitch = ld * es;
     const int64_t row_bytes = (int64_t)V * es;
+    const int64_t chunks = (row_bytes + 15) / 16 + 1;
+    const int G = chunks <= 72 ? 4 : chunks <= 144 ? 8 : chunks <= 288 ? 16 : 32;
+    const int rpw = 32 / G;
     const int smem_budget = 200 * 1024;
-    int warps = 0, stages = (o && o->stages > 0) ? o->stages : 3, R = 0;
-    if (stages < 2) stages = 2;
+    // One stage per warp and as many warps as fit hide the copy latency behind other warps'
+    // arithmetic and give the schedulers more independent work than a deeper ring with fewer
+    // warps does; a small matrix (a tile or two per warp) is better off prefetching.
+    const int64_t tiles_guess = N * row_pitch / 8192 + 1;
+    int warps = 0, R = 0;
+    int stages = (o && o->stages > 0) ? o->stages : (tiles_guess < 2ll * 24 * sm_count() ? 2 : 1);
+    if (stages < 1) stages = 1;
     if (stages > 8) stages = 8;
-    if (kernel != 1) {
-        const int cand[] = {16, 8, 4, 2, 1};
-        for (int w : cand) {
-            if (o && o->warps > 0 && o->warps != w) continue;
-            const int64_t per_stage = ((smem_budget - 1024) / ((int64_t)w * stages)) & ~127ll;
-            if (row_bytes + 48 > per_stage) continue;
-            warps = w;
-            int64_t r = 1 + (per_stage - 48 - row_bytes) / row_pitch;
-            if (r > 32) r = 32;
-            // a row pitch much wider than the row would drag the padding along: one row a tile
-            if (row_pitch > 2 * row_bytes) r = 1;
-            if (o && o->stage_bytes > 0 && o->stage_bytes < r) r = o->stage_bytes;
-            R = (int)r;
-            break;
+    int64_t stage_stride = 0;
+    if (kernel != 1 && row_pitch <= 2 * row_bytes + 64 && row_pitch < (1 << 20)) {
+        int64_t groups = 8192 / (rpw * row_pitch);
+        if (groups < 1) groups = 1;
+        if (o && o->stage_bytes > 0) groups = (o->stage_bytes + rpw - 1) / rpw;
+        for (; groups >= 1 && warps == 0; groups = groups > 1 ? groups / 2 : 0) {
+            R = (int)(groups * rpw);
+            stage_stride = ((R - 1) * row_pitch + row_bytes + 32 + 127) & ~127ll;
+            int64_t w = (smem_budget - 1024) / (stages * stage_stride);
+            if (w > 24) w = 24;
+            if (o && o->warps > 0 && o->warps < w) w = o->warps;
+            if (w >= 1) warps = (int)w;
         }
-        if (warps == 0) {
-            if (kernel == 2) return SSD_ERR_ARG;   // forced, but a row does not fit a stage
-            kernel = 1;
-        } else {
-            kernel = 2;
-        }
+    }
+    if (warps == 0) {
+        if (kernel == 2) return SSD_ERR_ARG;   // forced, but a row group does not fit a stage
+        kernel = 1;
+    } else {
+        kernel = 2;
     }
     cudaError_t e;
     if (o && o->ev_begin) {
@@ -507,14 +681,20 @@ int launch_ctc_rows(const void *logits, ssd_dtype dtype, int V, int64_t ld, int6
     }
     if (kernel == 2) {
         p.rows_per_tile = R; p.stages = stages; p.warps = warps;
-        p.stage_stride = (int)(((R - 1) * row_pitch + row_bytes + 32 + 127) & ~127ll);
+        p.stage_stride = (int)stage_stride;
         p.num_tiles = (N + R - 1) / R;
         const size_t smem = (size_t)((warps * stages * 8 + 127) & ~127) +
                             (size_t)warps * stages * p.stage_stride;
         int64_t ctas = (p.num_tiles + warps - 1) / warps;
         const int max_ctas = (o && o->ctas > 0) ? o->ctas : sm_count();
         if (ctas > max_ctas) ctas = max_ctas;
-        auto kern = dtype == SSD_F32 ? ctc_rows_tma<float> : ctc_rows_tma<bf16_t>;
+        void (*kern)(const CtcParams) = nullptr;
+        if (dtype == SSD_F32)
+            kern = G == 4 ? ctc_rows_tma<float, 4> : G == 8 ? ctc_rows_tma<float, 8>
+                 : G == 16 ? ctc_rows_tma<float, 16> : ctc_rows_tma<float, 32>;
+        else
+            kern = G == 4 ? ctc_rows_tma<bf16_t, 4> : G == 8 ? ctc_rows_tma<bf16_t, 8>
+                 : G == 16 ? ctc_rows_tma<bf16_t, 16> : ctc_rows_tma<bf16_t, 32>;
         e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
         kern<<<(unsigned)ctas, warps * 32, smem, L.stream>>>(p);
