@@ -309,6 +309,7 @@ template <typename T, int G>
 __global__ void __launch_bounds__(768, 1) ctc_rows_tma(const CtcParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     constexpr int ES = Elem<T>::kBytes;
+    pdl_enter();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int W = p.warps, S = p.stages, R = p.rows_per_tile;
     const int64_t gw = (int64_t)blockIdx.x * W + warp, GW = (int64_t)gridDim.x * W;
@@ -427,6 +428,7 @@ __global__ void __launch_bounds__(768, 1) ctc_rows_tma(const CtcParams p) {
 template <typename T>
 __global__ void __launch_bounds__(256) ctc_rows_plain(const CtcParams p) {
     constexpr int ES = Elem<T>::kBytes;
+    pdl_enter();
     const int lane = threadIdx.x & 31;
     const int64_t gw = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int64_t GW = ((int64_t)gridDim.x * blockDim.x) >> 5;
@@ -504,6 +506,7 @@ __global__ void __launch_bounds__(kUttThreads) collapse_kernel(
     __shared__ int warp_tot[32];
     __shared__ MaxAt scratch[32];
     __shared__ unsigned flags;
+    pdl_enter();
     const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nw = blockDim.x >> 5;
     const int64_t t0 = frame_off[b], t1 = frame_off[b + 1];
@@ -570,6 +573,7 @@ __global__ void __launch_bounds__(kUttThreads) gate_kernel(
     int32_t *__restrict__ argmax_frame) {
     __shared__ MaxAt scratch[32];
     __shared__ int not_below;
+    pdl_enter();
     const int b = blockIdx.x, tid = threadIdx.x;
     const int64_t t0 = frame_off[b], t1 = frame_off[b + 1];
     if (t0 < 0 || t1 < t0 || t1 > N) {
@@ -697,13 +701,15 @@ int launch_ctc_rows(const void *logits, ssd_dtype dtype, int V, int64_t ld, int6
                  : G == 16 ? ctc_rows_tma<bf16_t, 16> : ctc_rows_tma<bf16_t, 32>;
         e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
-        kern<<<(unsigned)ctas, warps * 32, smem, L.stream>>>(p);
+        e = launch_pdl(kern, (unsigned)ctas, (unsigned)(warps * 32), smem, L.stream, p);
+        if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
     } else {
         int64_t ctas = (N + 7) / 8;
         const int64_t cap = (o && o->ctas > 0) ? o->ctas : (int64_t)sm_count() * 8;
         if (ctas > cap) ctas = cap;
-        if (dtype == SSD_F32) ctc_rows_plain<float><<<(unsigned)ctas, 256, 0, L.stream>>>(p);
-        else ctc_rows_plain<bf16_t><<<(unsigned)ctas, 256, 0, L.stream>>>(p);
+        e = launch_pdl(dtype == SSD_F32 ? ctc_rows_plain<float> : ctc_rows_plain<bf16_t>,
+                       (unsigned)ctas, 256u, 0, L.stream, p);
+        if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
     }
     e = cudaGetLastError();
     if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
@@ -720,10 +726,10 @@ int launch_collapse(const int32_t *frame_argmax, const float *frame_entropy,
                     int32_t *draft_full_len, float *utt_max_entropy, uint32_t *utt_status,
                     cudaStream_t stream) {
     if (B == 0) return SSD_OK;
-    collapse_kernel<<<B, kUttThreads, 0, stream>>>(
+    cudaError_t e = launch_pdl(collapse_kernel, (unsigned)B, (unsigned)kUttThreads, 0, stream,
         frame_argmax, frame_entropy, frame_off, B, N, blank_id, max_draft_len, draft_tokens,
         draft_frames, draft_len, draft_full_len, utt_max_entropy, utt_status);
-    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
     return SSD_OK;
 }
@@ -732,9 +738,10 @@ int launch_gate(const float *frame_entropy, const int64_t *frame_off, int B, int
                 float tau, uint8_t *gate_accept, float *max_entropy, int32_t *argmax_frame,
                 cudaStream_t stream) {
     if (B == 0) return SSD_OK;
-    gate_kernel<<<B, kUttThreads, 0, stream>>>(frame_entropy, frame_off, B, N, tau, gate_accept,
-                                               max_entropy, argmax_frame);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_pdl(gate_kernel, (unsigned)B, (unsigned)kUttThreads, 0, stream,
+                               frame_entropy, frame_off, B, N, tau, gate_accept, max_entropy,
+                               argmax_frame);
+    if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
     return SSD_OK;
 }

@@ -148,6 +148,7 @@ template <typename T>
 __global__ void __launch_bounds__(544, 1) verify_rows_tma(const VerifyParams p) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     constexpr int ES = Elem<T>::kBytes, EPC = Elem<T>::kPerChunk;
+    pdl_enter();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int S = p.stages, CW = p.warps;
     // layout: full[S] | empty[S] | desc[S] | offsets cache | stages
@@ -313,6 +314,7 @@ __global__ void __launch_bounds__(544, 1) verify_rows_tma(const VerifyParams p) 
 template <typename T>
 __global__ void __launch_bounds__(256) verify_rows_plain(const VerifyParams p) {
     constexpr int ES = Elem<T>::kBytes;
+    pdl_enter();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
     for (int64_t item = blockIdx.x; item < p.num_items; item += gridDim.x) {
         const int64_t row = item / p.split;
@@ -351,6 +353,7 @@ __global__ void __launch_bounds__(kFinishThreads) verify_finish_kernel(
     constexpr int ES = Elem<T>::kBytes;
     __shared__ int first_reject;
     __shared__ unsigned flags;
+    pdl_enter();
     const int b = blockIdx.x, tid = threadIdx.x;
     const int64_t i0 = tok_off[b], i1 = tok_off[b + 1];
     const uint32_t internal = (*err_word == epoch) ? (uint32_t)SSD_UTT_INTERNAL : 0u;
@@ -499,11 +502,14 @@ int launch_verify(const void *logits, ssd_dtype dtype, int V, int64_t ld, int64_
             e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)plan.smem_bytes);
             if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
-            kern<<<(unsigned)ctas, (plan.warps + 1) * 32, plan.smem_bytes, L.stream>>>(p);
+            e = launch_pdl(kern, (unsigned)ctas, (unsigned)((plan.warps + 1) * 32), plan.smem_bytes,
+                           L.stream, p);
+            if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
         } else {
             ctas = p.num_items < 8ll * plan.ctas ? p.num_items : 8ll * plan.ctas;
-            if (dtype == SSD_F32) verify_rows_plain<float><<<(unsigned)ctas, 256, 0, L.stream>>>(p);
-            else verify_rows_plain<bf16_t><<<(unsigned)ctas, 256, 0, L.stream>>>(p);
+            e = launch_pdl(dtype == SSD_F32 ? verify_rows_plain<float> : verify_rows_plain<bf16_t>,
+                           (unsigned)ctas, 256u, 0, L.stream, p);
+            if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
         }
         e = cudaGetLastError();
         if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
@@ -515,16 +521,13 @@ int launch_verify(const void *logits, ssd_dtype dtype, int V, int64_t ld, int64_
     const double tau = (double)tau_slm;
     const int reject_none = !(tau > 0.0);
     const float log_tau = reject_none ? -INFINITY : (float)log(tau);
-    if (dtype == SSD_F32)
-        verify_finish_kernel<float><<<B, kFinishThreads, 0, L.stream>>>(
-            static_cast<const char *>(logits), V, ld, M, tok_off, draft_ids, B, log_tau,
-            reject_none, skip, partials, plan.partials, token_logp, row_lse, accepted_len,
-            all_accepted, utt_status, err_word, epoch);
-    else
-        verify_finish_kernel<bf16_t><<<B, kFinishThreads, 0, L.stream>>>(
-            static_cast<const char *>(logits), V, ld, M, tok_off, draft_ids, B, log_tau,
-            reject_none, skip, partials, plan.partials, token_logp, row_lse, accepted_len,
-            all_accepted, utt_status, err_word, epoch);
+    e = launch_pdl(dtype == SSD_F32 ? verify_finish_kernel<float> : verify_finish_kernel<bf16_t>,
+                   (unsigned)B, (unsigned)kFinishThreads, 0, L.stream,
+                   static_cast<const char *>(logits), V, ld, M, tok_off, draft_ids, B, log_tau,
+                   reject_none, skip, static_cast<const float2 *>(partials), plan.partials,
+                   token_logp, row_lse, accepted_len, all_accepted, utt_status,
+                   static_cast<const unsigned long long *>(err_word), epoch);
+    if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
     e = cudaGetLastError();
     if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
     return SSD_OK;
