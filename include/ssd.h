@@ -45,7 +45,8 @@ enum {
     SSD_ERR_DTYPE = 3,     /* dtype is neither SSD_F32 nor SSD_BF16 */
     SSD_ERR_WORKSPACE = 4, /* workspace NULL or smaller than the *_workspace_bytes() answer */
     SSD_ERR_CUDA = 5,      /* a CUDA runtime call failed; see ssd_last_cuda_error() */
-    SSD_ERR_ALIGN = 6      /* logits base not aligned to the element size */
+    SSD_ERR_ALIGN = 6,     /* logits base not aligned to the element size */
+    SSD_ERR_TOO_LARGE = 7  /* ssd_verify_static: the sizes need more scratch than its fixed array */
 };
 
 /* bits of utt_status[b] */
@@ -173,6 +174,47 @@ int32_t ssd_verify(const void *logits, ssd_dtype dtype, int32_t V, int64_t ld,
                    int32_t *accepted_len, uint8_t *all_accepted, uint32_t *utt_status,
                    void *workspace, size_t workspace_bytes, void *stream,
                    const ssd_launch_opts *opts);
+
+/*
+ * ssd_verify without a workspace argument, for callers that cannot allocate device memory.
+ * (The paper has no counterpart: this is a packaging variant of ssd_verify, same arithmetic.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a region the host
+ * framework forbids allocation in (a real-time audio callback, a plugin sandbox that hands out
+ * only the buffers it owns, an embedding runtime whose memory is carved up before start-up), or
+ * simply a caller that has no allocator of its own and does not want to size a workspace.
+ * ssd_verify asks such a caller for scratch it has no means to provide; this call brings its own.
+ *
+ * The scratch is a fixed array of SSD_VERIFY_STATIC_SCRATCH_BYTES inside the library's device
+ * image.  Every device that loads the library holds that much memory until the process exits,
+ * whether or not this function is ever called.  The call itself allocates and frees nothing
+ * (no cudaMalloc, no cudaFree, no allocating library routine); inputs and outputs are still
+ * the caller's buffers, exactly as for ssd_verify, and the results are the same.
+ *
+ * Limit: sizes for which ssd_verify_workspace_bytes(B, M, V, dtype, opts) exceeds
+ * SSD_VERIFY_STATIC_SCRATCH_BYTES are refused with SSD_ERR_TOO_LARGE before anything is
+ * enqueued (with the default options the scratch is 128 bytes per logits row plus a header, so
+ * about 65,000 rows fit; few rows of a wide vocabulary use more per row and still fit).
+ *
+ * First call on a device: the function looks up the device address of the array (once per
+ * device, under a lock, with the caller's current device).  Make that first call outside any
+ * stream capture.  Later calls only read the cached address.
+ *
+ * Sharing: all calls on a device use the same array and it keeps whatever the last call left
+ * in it.  Nothing in it needs clearing between calls.  Two calls whose kernels can run at the
+ * same time on one device (different streams, or different host threads on different streams)
+ * overwrite each other's partial sums: keep calls to this function on a device in one stream,
+ * or otherwise ordered.
+ *
+ * Errors: those of ssd_verify except SSD_ERR_WORKSPACE, plus SSD_ERR_TOO_LARGE.
+ */
+#define SSD_VERIFY_STATIC_SCRATCH_BYTES (8u << 20)
+int32_t ssd_verify_static(const void *logits, ssd_dtype dtype, int32_t V, int64_t ld,
+                          const int64_t *tok_off, const int32_t *draft_ids, int32_t B, int64_t M,
+                          float tau_slm, const uint8_t *skip,
+                          float *token_logp, float *row_lse,
+                          int32_t *accepted_len, uint8_t *all_accepted, uint32_t *utt_status,
+                          void *stream, const ssd_launch_opts *opts);
 
 #ifdef __cplusplus
 }

@@ -13,7 +13,8 @@ import torch
 
 F32, BF16 = 0, 1
 UTT_NONFINITE, UTT_BAD_DRAFT_ID, UTT_BAD_OFFSETS, UTT_INTERNAL = 1, 2, 4, 0x80000000
-OK, ERR_NULL, ERR_ARG, ERR_DTYPE, ERR_WORKSPACE, ERR_CUDA, ERR_ALIGN = range(7)
+OK, ERR_NULL, ERR_ARG, ERR_DTYPE, ERR_WORKSPACE, ERR_CUDA, ERR_ALIGN, ERR_TOO_LARGE = range(8)
+VERIFY_STATIC_SCRATCH_BYTES = 8 << 20
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libssd.so")
@@ -63,6 +64,9 @@ def lib():
         L.ssd_verify.restype = i32
         L.ssd_verify.argtypes = [vp, C.c_int, i32, i64, vp, vp, i32, i64, C.c_float, vp,
                                  vp, vp, vp, vp, vp, vp, C.c_size_t, vp, vp]
+        L.ssd_verify_static.restype = i32
+        L.ssd_verify_static.argtypes = [vp, C.c_int, i32, i64, vp, vp, i32, i64, C.c_float, vp,
+                                        vp, vp, vp, vp, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -200,6 +204,32 @@ def ssd_verify(logits: torch.Tensor, tok_off: torch.Tensor, draft_ids: torch.Ten
         _opts(opts))
     if rc != OK:
         raise SsdError(rc, "ssd_verify")
+    return out
+
+
+def ssd_verify_static(logits: torch.Tensor, tok_off: torch.Tensor, draft_ids: torch.Tensor,
+                      tau_slm: float, out: Dict[str, torch.Tensor],
+                      skip: Optional[torch.Tensor] = None, V: Optional[int] = None,
+                      opts: Optional[LaunchOpts] = None) -> Dict[str, torch.Tensor]:
+    """ssd_verify for callers that cannot allocate: the scratch is the library's own fixed
+    device array, so `out` holds only the result tensors (token_logp, row_lse, accepted_len,
+    all_accepted, utt_status), which the caller owns and must pass in.  This wrapper allocates
+    nothing either.  Sizes beyond the fixed array raise SsdError with code ERR_TOO_LARGE."""
+    M, ld = _rows_ld(logits)
+    V = logits.shape[1] if V is None else V
+    B = tok_off.shape[0] - 1
+    if tok_off.dtype != torch.int64 or draft_ids.dtype != torch.int32:
+        raise TypeError("tok_off must be int64 and draft_ids int32")
+    if skip is not None and skip.dtype != torch.uint8:
+        raise TypeError("skip must be uint8")
+    rc = lib().ssd_verify_static(
+        _dev(logits, "logits"), _dtype_code(logits), V, ld, _dev(tok_off, "tok_off"),
+        _dev(draft_ids, "draft_ids"), B, M, C.c_float(tau_slm), _dev(skip, "skip"),
+        _dev(out["token_logp"], "token_logp"), _dev(out.get("row_lse"), "row_lse"),
+        _dev(out["accepted_len"], "accepted_len"), _dev(out["all_accepted"], "all_accepted"),
+        _dev(out["utt_status"], "utt_status"), _stream(), _opts(opts))
+    if rc != OK:
+        raise SsdError(rc, "ssd_verify_static")
     return out
 
 

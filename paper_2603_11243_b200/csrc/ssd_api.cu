@@ -20,6 +20,8 @@ const char *ssd_status_string(int32_t status) {
         case SSD_ERR_WORKSPACE: return "SSD_ERR_WORKSPACE: workspace missing, misaligned or too small";
         case SSD_ERR_CUDA: return "SSD_ERR_CUDA: a CUDA runtime call failed";
         case SSD_ERR_ALIGN: return "SSD_ERR_ALIGN: logits not aligned to the element size";
+        case SSD_ERR_TOO_LARGE:
+            return "SSD_ERR_TOO_LARGE: the sizes need more scratch than ssd_verify_static's fixed array";
         default: return "unknown status";
     }
 }
