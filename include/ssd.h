@@ -72,6 +72,9 @@ typedef struct ssd_launch_opts {
     int32_t split;        /* verify: column spans per logits row */
     void *ev_begin;       /* cudaEvent_t recorded just before the streaming kernel, or NULL */
     void *ev_end;         /* cudaEvent_t recorded just after the streaming kernel, or NULL */
+    int32_t fma_exp;      /* verify, bf16: pairs of exponentials per 16-byte chunk evaluated by a
+                             polynomial on the FMA pipe instead of the special-function unit:
+                             0 auto; 1..3 that many of the 4 pairs; -1 none */
 } ssd_launch_opts;
 
 /* Human-readable name of a return code (static storage). */

@@ -33,7 +33,7 @@ class LaunchOpts(C.Structure):
     """Mirror of ssd_launch_opts (include/ssd.h)."""
     _fields_ = [("kernel", C.c_int32), ("ctas", C.c_int32), ("warps", C.c_int32),
                 ("stages", C.c_int32), ("stage_bytes", C.c_int32), ("split", C.c_int32),
-                ("ev_begin", C.c_void_p), ("ev_end", C.c_void_p)]
+                ("ev_begin", C.c_void_p), ("ev_end", C.c_void_p), ("fma_exp", C.c_int32)]
 
 
 _lib = None

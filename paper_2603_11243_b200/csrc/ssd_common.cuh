@@ -187,6 +187,35 @@ __device__ __forceinline__ float2 bf16x2_add_f32(uint32_t w, float c) {
     return d;
 }
 
+__device__ __forceinline__ float fmax_nan_fwd(float a, float b) {
+    float d;
+    asm("max.NaN.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+    return d;
+}
+
+// 2^t for a pair, on the FMA pipe: round t to the nearest integer n with the 1.5*2^23 trick,
+// evaluate a degree-4 polynomial for 2^f on f = t - n in [-1/2, 1/2] (relative error 3.6e-6)
+// and add n to the exponent field.  t is clamped to >= -126 first (the result is then at most
+// 2^-126 where the true value is smaller), NaN is kept by the clamp; t >= 128 or NaN give a
+// non-finite or huge value that the callers' range checks catch.
+__device__ __forceinline__ float2 exp2_fma_pair(float2 t) {
+    const float kMagic = 12582912.f;
+    t.x = fmax_nan_fwd(t.x, -126.f);
+    t.y = fmax_nan_fwd(t.y, -126.f);
+    const float2 r = fadd2(t, make_float2(kMagic, kMagic));
+    const float2 n = fadd2(r, make_float2(-kMagic, -kMagic));
+    const float2 f = ffma2(n, make_float2(-1.f, -1.f), t);
+    float2 p = make_float2(0.00966636836528778f, 0.00966636836528778f);
+    p = ffma2(p, f, make_float2(0.055921975523233414f, 0.055921975523233414f));
+    p = ffma2(p, f, make_float2(0.2402234971523285f, 0.2402234971523285f));
+    p = ffma2(p, f, make_float2(0.6931210160255432f, 0.6931210160255432f));
+    p = ffma2(p, f, make_float2(1.0f, 1.0f));
+    float2 y;
+    y.x = __int_as_float(__float_as_int(r.x) * (1 << 23) + __float_as_int(p.x));
+    y.y = __int_as_float(__float_as_int(r.y) * (1 << 23) + __float_as_int(p.y));
+    return y;
+}
+
 // order-preserving map float -> int32 (for integer warp reductions of float maxima)
 __device__ __forceinline__ int32_t float_key(float f) {
     int32_t b = __float_as_int(f);
@@ -298,6 +327,7 @@ struct VerifyPlan {
     int stages;
     int stage_bytes;
     int split;         // column spans per row
+    int fma_exp;       // pairs per chunk whose exponential runs on the FMA pipe (bf16 only)
     int partials;      // partial (max, sum) pairs per row = split * warps
     size_t smem_bytes;
     size_t workspace_bytes;

@@ -77,43 +77,59 @@ __device__ __forceinline__ float2 exp2_pair(float2 x, float2 scale, float2 nmh) 
     const float2 t = ffma2(x, scale, nmh);
     return make_float2(ex2(t.x), ex2(t.y));
 }
-
-template <typename T> __device__ __forceinline__ void add_chunk(const uint4 &w, float nmh, Online &st);
-template <> __device__ __forceinline__ void add_chunk<float>(const uint4 &w, float nmh, Online &st) {
-    const float2 sc = make_float2(kLog2e, kLog2e), nm = make_float2(nmh, nmh);
-    st.Sa = fadd2(st.Sa, exp2_pair(make_float2(__uint_as_float(w.x), __uint_as_float(w.y)), sc, nm));
-    st.Sb = fadd2(st.Sb, exp2_pair(make_float2(__uint_as_float(w.z), __uint_as_float(w.w)), sc, nm));
+__device__ __forceinline__ float2 exp2_pair_fma(float2 x, float2 scale, float2 nmh) {
+    return exp2_fma_pair(ffma2(x, scale, nmh));
 }
-template <> __device__ __forceinline__ void add_chunk<bf16_t>(const uint4 &w, float nmh, Online &st) {
+
+// kF of the 4 pairs of a bf16 chunk take the FMA-pipe exponential: the special-function unit
+// (16 results per clock per SM) is what bounds this kernel for bf16 logits, and the FMA pipe
+// has slots to spare.
+template <typename T, int kF>
+__device__ __forceinline__ void add_chunk(const uint4 &w, float nmh, Online &st) {
     const float2 sc = make_float2(kLog2e, kLog2e), nm = make_float2(nmh, nmh);
-    st.Sa = fadd2(st.Sa, exp2_pair(make_float2(bf16_lo(w.x), bf16_hi(w.x)), sc, nm));
-    st.Sb = fadd2(st.Sb, exp2_pair(make_float2(bf16_lo(w.y), bf16_hi(w.y)), sc, nm));
-    st.Sa = fadd2(st.Sa, exp2_pair(make_float2(bf16_lo(w.z), bf16_hi(w.z)), sc, nm));
-    st.Sb = fadd2(st.Sb, exp2_pair(make_float2(bf16_lo(w.w), bf16_hi(w.w)), sc, nm));
+    if (Elem<T>::kBytes == 4) {
+        st.Sa = fadd2(st.Sa, exp2_pair(make_float2(__uint_as_float(w.x), __uint_as_float(w.y)), sc, nm));
+        st.Sb = fadd2(st.Sb, exp2_pair(make_float2(__uint_as_float(w.z), __uint_as_float(w.w)), sc, nm));
+    } else {
+        const float2 x0 = make_float2(bf16_lo(w.x), bf16_hi(w.x)), x1 = make_float2(bf16_lo(w.y), bf16_hi(w.y));
+        const float2 x2 = make_float2(bf16_lo(w.z), bf16_hi(w.z)), x3 = make_float2(bf16_lo(w.w), bf16_hi(w.w));
+        st.Sa = fadd2(st.Sa, kF >= 1 ? exp2_pair_fma(x0, sc, nm) : exp2_pair(x0, sc, nm));
+        st.Sb = fadd2(st.Sb, kF >= 3 ? exp2_pair_fma(x1, sc, nm) : exp2_pair(x1, sc, nm));
+        st.Sa = fadd2(st.Sa, kF >= 2 ? exp2_pair_fma(x2, sc, nm) : exp2_pair(x2, sc, nm));
+        st.Sb = fadd2(st.Sb, exp2_pair(x3, sc, nm));
+    }
 }
 
 // Adds this thread's chunks (ct, ct + NT, ...) of a stage holding n chunks to its running sum.
-template <typename T>
+// Four chunks are fetched before any is used; the last, partial group of up to three is fetched
+// together as well.
+template <typename T, int kF>
 __device__ __forceinline__ void add_chunks(uint32_t a0, int n, int ct, int NT, Online &st) {
     const float nmh = -st.mh;
+    const uint32_t step = (uint32_t)NT * 16;
+    uint32_t a = a0 + (uint32_t)ct * 16;
     int c = ct;
-    for (; c + 3 * NT < n; c += 4 * NT) {
-        const uint4 w0 = lds128(a0 + (uint32_t)c * 16);
-        const uint4 w1 = lds128(a0 + (uint32_t)(c + NT) * 16);
-        const uint4 w2 = lds128(a0 + (uint32_t)(c + 2 * NT) * 16);
-        const uint4 w3 = lds128(a0 + (uint32_t)(c + 3 * NT) * 16);
-        add_chunk<T>(w0, nmh, st);
-        add_chunk<T>(w1, nmh, st);
-        add_chunk<T>(w2, nmh, st);
-        add_chunk<T>(w3, nmh, st);
+    for (; c + 3 * NT < n; c += 4 * NT, a += 4 * step) {
+        const uint4 w0 = lds128(a), w1 = lds128(a + step), w2 = lds128(a + 2 * step),
+                    w3 = lds128(a + 3 * step);
+        add_chunk<T, kF>(w0, nmh, st);
+        add_chunk<T, kF>(w1, nmh, st);
+        add_chunk<T, kF>(w2, nmh, st);
+        add_chunk<T, kF>(w3, nmh, st);
     }
-    for (; c < n; c += NT) {
-        const uint4 w = lds128(a0 + (uint32_t)c * 16);
-        add_chunk<T>(w, nmh, st);
+    if (c < n) {
+        const bool h1 = c + NT < n, h2 = c + 2 * NT < n;
+        const uint4 w0 = lds128(a);
+        uint4 w1 = w0, w2 = w0;
+        if (h1) w1 = lds128(a + step);
+        if (h2) w2 = lds128(a + 2 * step);
+        add_chunk<T, kF>(w0, nmh, st);
+        if (h1) add_chunk<T, kF>(w1, nmh, st);
+        if (h2) add_chunk<T, kF>(w2, nmh, st);
     }
 }
 
-template <typename T>
+template <typename T, int kF>
 __device__ __forceinline__ void consume_stage(uint32_t a0, int n, int ct, int NT, Online &st) {
     if (ct >= n) return;
     if (!(st.m > -INFINITY)) {
@@ -122,7 +138,7 @@ __device__ __forceinline__ void consume_stage(uint32_t a0, int n, int ct, int NT
         if (cm > -INFINITY) { st.m = cm; st.mh = cm * kLog2e; }
     }
     const Online saved = st;
-    add_chunks<T>(a0, n, ct, NT, st);
+    add_chunks<T, kF>(a0, n, ct, NT, st);
     if (!(st.total() < kSumLimit)) {
         // an element far above the reference, a NaN or +inf, or only -inf so far: redo the
         // stage relative to the maximum of this thread's chunks
@@ -130,7 +146,7 @@ __device__ __forceinline__ void consume_stage(uint32_t a0, int n, int ct, int NT
         float cm = -INFINITY;
         for (int c = ct; c < n; c += NT) cm = fmaxf(cm, chunk_max<T>(lds128(a0 + (uint32_t)c * 16)));
         if (cm > st.m) st.raise_to(cm);
-        if (st.m > -INFINITY) add_chunks<T>(a0, n, ct, NT, st);
+        if (st.m > -INFINITY) add_chunks<T, kF>(a0, n, ct, NT, st);
     }
 }
 
@@ -144,7 +160,7 @@ __device__ __forceinline__ float2 warp_merge(const Online &st) {
     return make_float2(M, Sw);
 }
 
-template <typename T>
+template <typename T, int kF>
 __global__ void __launch_bounds__(544, 1) verify_rows_tma(const VerifyParams p) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     constexpr int ES = Elem<T>::kBytes, EPC = Elem<T>::kPerChunk;
@@ -292,7 +308,7 @@ __global__ void __launch_bounds__(544, 1) verify_rows_tma(const VerifyParams p) 
             const int n = desc[s].nchunks;
             const uint32_t flags = desc[s].flags;
             if (flags & kFlagEnd) break;
-            consume_stage<T>(stage0 + (uint32_t)s * p.stage_bytes, n, ct, NT, st);
+            consume_stage<T, kF>(stage0 + (uint32_t)s * p.stage_bytes, n, ct, NT, st);
             int64_t slot = 0;
             if (flags & kFlagLast) slot = desc[s].slot;
             __syncwarp();
@@ -439,7 +455,7 @@ int plan_verify(int B, int64_t M, int V, ssd_dtype dtype, const ssd_launch_opts 
     if (split > 64) split = 64;
     pl.split = split;
     if (pl.kernel == 2) {
-        pl.warps = (o && o->warps > 0) ? o->warps : 16;
+        pl.warps = (o && o->warps > 0) ? o->warps : (row_bytes >= 96 * 1024 ? 12 : 16);
         if (pl.warps > 16) return SSD_ERR_ARG;
         if (o && o->stage_bytes > 0) {
             pl.stage_bytes = o->stage_bytes;
@@ -467,6 +483,10 @@ int plan_verify(int B, int64_t M, int V, ssd_dtype dtype, const ssd_launch_opts 
         pl.warps = 8;
         pl.stages = 0; pl.stage_bytes = 0; pl.smem_bytes = 0;
     }
+    // measured: one pair of four on the FMA pipe is the best split for bf16 (two lose to
+    // instruction issue); fp32 logits are HBM-bound without it
+    pl.fma_exp = (o && o->fma_exp) ? (o->fma_exp < 0 ? 0 : o->fma_exp) : (dtype == SSD_BF16 ? 1 : 0);
+    if (pl.fma_exp > 3) return SSD_ERR_ARG;
     pl.partials = split * pl.warps;
     pl.workspace_bytes = 256 + (size_t)M * pl.partials * sizeof(float2);
     *plan = pl;
@@ -498,7 +518,11 @@ int launch_verify(const void *logits, ssd_dtype dtype, int V, int64_t ld, int64_
             if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
         }
         if (plan.kernel == 2) {
-            auto kern = dtype == SSD_F32 ? verify_rows_tma<float> : verify_rows_tma<bf16_t>;
+            void (*kern)(const VerifyParams) = verify_rows_tma<float, 0>;
+            if (dtype == SSD_BF16)
+                kern = plan.fma_exp == 1 ? verify_rows_tma<bf16_t, 1>
+                     : plan.fma_exp == 2 ? verify_rows_tma<bf16_t, 2>
+                     : plan.fma_exp == 3 ? verify_rows_tma<bf16_t, 3> : verify_rows_tma<bf16_t, 0>;
             e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)plan.smem_bytes);
             if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
