@@ -45,6 +45,10 @@ def parse_args():
     ap.add_argument("--config", type=int, default=1, help="workload index (1..3)")
     ap.add_argument("--e2e-steps", type=int, default=30)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", default=None, metavar="FILE",
+                    help="time every point of the throughput sweep (configuration 4) and write one "
+                         "JSON line per point to FILE instead of the benchmark line")
+    ap.add_argument("--sweep-filter", default="", help="only points whose name contains this")
     ap.add_argument("--ncu-small", action="store_true",
                     help="profiling aid: one input set, no end-to-end leg, no CPU baseline")
     return ap.parse_args()
@@ -472,8 +476,104 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+# ---- the throughput sweep ------------------------------------------------------------------
+SWEEP_B = (1, 8, 64, 256, 1024)
+SWEEP_V = (32000, 49152, 100352, 152064)
+SWEEP_DTYPES = ("f32", "bf16")
+SWEEP_MAX_RESIDENT = 48e9        # bytes of logits generated at a time; larger points run as
+                                 # equal sub-batches, each timed on its own, times added
+
+
+def time_steps(sets, steps, warmup, every=3):
+    """Mean step time and mean streaming-kernel times (ms) over `steps` steps."""
+    import torch
+    from paper_2603_11243_b200 import binding as ssd
+    n_sets = len(sets)
+
+    def step(s, o_ctc=None, o_ver=None):
+        s["call_ctc"](o_ctc)
+        s["call_gate"]()
+        s["call_verify"](o_ver)
+
+    for i in range(warmup):
+        step(sets[i % n_sets])
+    timed = list(range(0, steps, every))
+    ev = make_events(4 * len(timed) + 2)
+    opts = {}
+    for j, i in enumerate(timed):
+        a, b = ssd.LaunchOpts(), ssd.LaunchOpts()
+        a.ev_begin, a.ev_end = ev[4 * j].cuda_event, ev[4 * j + 1].cuda_event
+        b.ev_begin, b.ev_end = ev[4 * j + 2].cuda_event, ev[4 * j + 3].cuda_event
+        opts[i] = (a, b)
+    torch.cuda.synchronize()
+    ev[-2].record()
+    for i in range(steps):
+        o = opts.get(i, (None, None))
+        step(sets[i % n_sets], o[0], o[1])
+    ev[-1].record()
+    torch.cuda.synchronize()
+    t_ctc = statistics.mean(ev[4 * j].elapsed_time(ev[4 * j + 1]) for j in range(len(timed)))
+    t_ver = statistics.mean(ev[4 * j + 2].elapsed_time(ev[4 * j + 3]) for j in range(len(timed)))
+    return ev[-2].elapsed_time(ev[-1]) / steps, t_ctc, t_ver
+
+
+def run_sweep(args):
+    import torch
+    from paper_2603_11243_b200 import build as lib_build
+    from paper_2603_11243_b200 import synth
+    lib_build.build()
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    peak, peak_kind = peaks()
+    with open(args.sweep, "a") as out:
+        for dtype in SWEEP_DTYPES:
+            for V in SWEEP_V:
+                for B in SWEEP_B:
+                    w = synth.sweep_point(B, V, dtype)
+                    if args.sweep_filter and args.sweep_filter not in w.name:
+                        continue
+                    es = 2 if dtype == "bf16" else 4
+                    est = B * (1000 * w.V_ctc + 250 * V) * es
+                    n_sub = max(1, math.ceil(est / SWEEP_MAX_RESIDENT))
+                    while B % n_sub:
+                        n_sub += 1
+                    n_sets = max(1, min(8, math.ceil(4e8 / (est / n_sub))))
+                    steps = int(max(10, min(300, 0.25 / (est / n_sub / 5e12))))
+                    ms = t_ctc = t_ver = 0.0
+                    ctc_b = ver_b = 0
+                    for sub in range(n_sub):
+                        ws = synth.scaled(w, B=B // n_sub, seed=w.seed + 31 * sub)
+                        sets = build_sets(ws, device, n_sets)
+                        a, b, c = time_steps(sets, steps, 5)
+                        ms, t_ctc, t_ver = ms + a, t_ctc + b, t_ver + c
+                        ctc_b += sets[0]["ctc_bytes"]
+                        ver_b += sets[0]["verify_bytes"]
+                        del sets
+                        torch.cuda.empty_cache()
+                    nbytes = ctc_b + ver_b
+                    line = {"point": w.name, "B": B, "V_llm": V, "dtype": dtype,
+                            "sub_batches": n_sub, "input_sets": n_sets, "steps": steps,
+                            "logits_bytes": nbytes, "ms_per_step": round(ms, 5),
+                            "utterances_per_s": round(B / (ms * 1e-3), 1),
+                            "step_gbs": round(nbytes / (ms * 1e-3) / 1e9, 1),
+                            "step_frac": round(nbytes / (ms * 1e-3) / 1e9 / peak, 4),
+                            "ctc_us": round(t_ctc * 1e3, 2),
+                            "ctc_gbs": round(ctc_b / (t_ctc * 1e-3) / 1e9, 1),
+                            "ctc_frac": round(ctc_b / (t_ctc * 1e-3) / 1e9 / peak, 4),
+                            "verify_us": round(t_ver * 1e3, 2),
+                            "verify_gbs": round(ver_b / (t_ver * 1e-3) / 1e9, 1) if t_ver else None,
+                            "verify_frac": round(ver_b / (t_ver * 1e-3) / 1e9 / peak, 4) if t_ver else None,
+                            "peak_gbs": peak, "peak_kind": peak_kind}
+                    out.write(json.dumps(line) + "\n")
+                    out.flush()
+                    print(json.dumps(line), flush=True)
+
+
 def main():
     args = parse_args()
+    if args.sweep:
+        run_sweep(args)
+        return
     if args.impl == "reference":
         run_reference(args)
         return

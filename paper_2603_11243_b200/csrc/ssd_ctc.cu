@@ -469,7 +469,9 @@ __global__ void __launch_bounds__(256) ctc_rows_plain(const CtcParams p) {
 }
 
 // ---- collapse B and per-utterance maximum entropy: one CTA per utterance ----------------------
-constexpr int kUttThreads = 256;
+// These kernels are chains of a few dependent memory round trips; a wide CTA takes an utterance
+// of up to 1024 frames in one sweep, and the loads of a sweep are issued together.
+constexpr int kUttThreads = 1024;
 
 struct MaxAt {
     float v;
@@ -480,8 +482,7 @@ __device__ __forceinline__ MaxAt better(MaxAt a, MaxAt b) {
     if (b.at >= 0 && (a.at < 0 || b.v > a.v || (b.v == a.v && b.at < a.at))) return b;
     return a;
 }
-__device__ MaxAt block_max_at(MaxAt x, MaxAt *scratch /* [32] shared */) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+__device__ __forceinline__ MaxAt warp_max_at(MaxAt x) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         MaxAt y;
@@ -489,11 +490,19 @@ __device__ MaxAt block_max_at(MaxAt x, MaxAt *scratch /* [32] shared */) {
         y.at = __shfl_xor_sync(0xffffffffu, x.at, o);
         x = better(x, y);
     }
-    __syncthreads();
+    return x;
+}
+// Maximum over the block; valid in warp 0 (all its lanes).  One __syncthreads.
+__device__ __forceinline__ MaxAt block_max_at(MaxAt x, MaxAt *scratch /* [32] shared */) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    x = warp_max_at(x);
     if (lane == 0) scratch[warp] = x;
     __syncthreads();
-    MaxAt r = scratch[0];
-    for (int w = 1; w < nw; ++w) r = better(r, scratch[w]);
+    MaxAt r{0.f, -1};
+    if (warp == 0) {
+        if (lane < nw) r = scratch[lane];
+        r = warp_max_at(r);
+    }
     return r;
 }
 
@@ -503,9 +512,9 @@ __global__ void __launch_bounds__(kUttThreads) collapse_kernel(
     int32_t *__restrict__ draft_tokens, int32_t *__restrict__ draft_frames,
     int32_t *__restrict__ draft_len, int32_t *__restrict__ draft_full_len,
     float *__restrict__ utt_max_entropy, uint32_t *__restrict__ utt_status) {
-    __shared__ int warp_tot[32];
+    __shared__ int warp_tot[2][32];
     __shared__ MaxAt scratch[32];
-    __shared__ unsigned flags;
+    __shared__ unsigned flags_sh[32];
     pdl_enter();
     const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nw = blockDim.x >> 5;
@@ -517,20 +526,23 @@ __global__ void __launch_bounds__(kUttThreads) collapse_kernel(
         }
         return;
     }
-    if (tid == 0) flags = 0;
-    __syncthreads();
     const int64_t T = t1 - t0;
-    int base = 0;
+    int base = 0, buf = 0;
     MaxAt best{0.f, -1};
     unsigned myflags = 0;
-    for (int64_t tile = 0; tile < T; tile += blockDim.x) {
+    for (int64_t tile = 0; tile < T; tile += blockDim.x, buf ^= 1) {
         const int64_t t = tile + tid;
         const bool valid = t < T;
-        int a = blank_id, prev = -1;
+        int a = blank_id;
+        float h = 0.f;
         if (valid) {
             a = frame_argmax[t0 + t];
-            if (t > 0) prev = frame_argmax[t0 + t - 1];
-            const float h = frame_entropy[t0 + t];
+            h = frame_entropy[t0 + t];
+        }
+        // the previous frame's symbol: the neighbouring lane has it, except for lane 0
+        int prev = __shfl_up_sync(0xffffffffu, a, 1);
+        if (lane == 0) prev = (valid && t > 0) ? frame_argmax[t0 + t - 1] : -1;
+        if (valid) {
             if (h != h) {
                 myflags |= (__float_as_uint(h) == kNanInternal) ? SSD_UTT_INTERNAL : SSD_UTT_NONFINITE;
             } else {
@@ -540,15 +552,18 @@ __global__ void __launch_bounds__(kUttThreads) collapse_kernel(
         const bool keep = valid && a != blank_id && (t == 0 || a != prev);
         const unsigned bal = __ballot_sync(0xffffffffu, keep);
         const int prefix = __popc(bal & ((1u << lane) - 1));
-        __syncthreads();                       // previous tile's totals fully consumed
-        if (lane == 0) warp_tot[warp] = __popc(bal);
-        __syncthreads();
-        int before = 0, total = 0;
-        for (int w = 0; w < nw; ++w) {
-            const int c = warp_tot[w];
-            if (w < warp) before += c;
-            total += c;
+        if (lane == 0) warp_tot[buf][warp] = __popc(bal);
+        __syncthreads();                       // the other buffer is free again after this
+        // every warp scans the (at most 32) warp totals by itself
+        const int mine = lane < nw ? warp_tot[buf][lane] : 0;
+        int incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int y = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += y;
         }
+        const int before = __shfl_sync(0xffffffffu, incl - mine, warp);
+        const int total = __shfl_sync(0xffffffffu, incl, 31);
         const int pos = base + before + prefix;
         if (keep && pos < cap) {
             draft_tokens[t0 + pos] = a;
@@ -556,14 +571,18 @@ __global__ void __launch_bounds__(kUttThreads) collapse_kernel(
         }
         base += total;
     }
-    best = block_max_at(best, scratch);
-    if (myflags) atomicOr(&flags, myflags);
-    __syncthreads();
-    if (tid == 0) {
-        draft_full_len[b] = base;
-        draft_len[b] = min(base, cap);
-        utt_max_entropy[b] = best.at >= 0 ? best.v : 0.f;
-        utt_status[b] = flags;
+    myflags = __reduce_or_sync(0xffffffffu, myflags);
+    if (lane == 0) flags_sh[warp] = myflags;
+    best = block_max_at(best, scratch);        // __syncthreads inside: flags_sh visible after it
+    if (warp == 0) {
+        unsigned f = lane < nw ? flags_sh[lane] : 0u;
+        f = __reduce_or_sync(0xffffffffu, f);
+        if (lane == 0) {
+            draft_full_len[b] = base;
+            draft_len[b] = min(base, cap);
+            utt_max_entropy[b] = best.at >= 0 ? best.v : 0.f;
+            utt_status[b] = f;
+        }
     }
 }
 
@@ -572,9 +591,10 @@ __global__ void __launch_bounds__(kUttThreads) gate_kernel(
     int64_t N, float tau, uint8_t *__restrict__ gate_accept, float *__restrict__ max_entropy,
     int32_t *__restrict__ argmax_frame) {
     __shared__ MaxAt scratch[32];
-    __shared__ int not_below;
+    __shared__ int bad_sh[32];
     pdl_enter();
-    const int b = blockIdx.x, tid = threadIdx.x;
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nw = blockDim.x >> 5;
     const int64_t t0 = frame_off[b], t1 = frame_off[b + 1];
     if (t0 < 0 || t1 < t0 || t1 > N) {
         if (tid == 0) {
@@ -583,8 +603,6 @@ __global__ void __launch_bounds__(kUttThreads) gate_kernel(
         }
         return;
     }
-    if (tid == 0) not_below = 0;
-    __syncthreads();
     const int64_t T = t1 - t0;
     MaxAt best{0.f, -1};
     int bad = 0;
@@ -593,13 +611,17 @@ __global__ void __launch_bounds__(kUttThreads) gate_kernel(
         if (!(h < tau)) bad = 1;             // Eq. 3 is strict; NaN never passes
         if (h == h) best = better(best, MaxAt{h, (int)t});
     }
-    if (bad) atomicOr(&not_below, 1);
-    best = block_max_at(best, scratch);       // contains __syncthreads
-    if (tid == 0) {
-        const bool accept = (T == 0) ? (0.f < tau) : (not_below == 0);
-        gate_accept[b] = accept ? 1 : 0;
-        max_entropy[b] = best.at >= 0 ? best.v : 0.f;
-        if (argmax_frame) argmax_frame[b] = best.at;
+    bad = __any_sync(0xffffffffu, bad);
+    if (lane == 0) bad_sh[warp] = bad;
+    best = block_max_at(best, scratch);       // __syncthreads inside
+    if (warp == 0) {
+        const int any_bad = __any_sync(0xffffffffu, lane < nw ? bad_sh[lane] : 0);
+        if (lane == 0) {
+            const bool accept = (T == 0) ? (0.f < tau) : !any_bad;
+            gate_accept[b] = accept ? 1 : 0;
+            max_entropy[b] = best.at >= 0 ? best.v : 0.f;
+            if (argmax_frame) argmax_frame[b] = best.at;
+        }
     }
 }
 

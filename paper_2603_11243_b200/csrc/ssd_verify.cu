@@ -355,7 +355,7 @@ __global__ void __launch_bounds__(256) verify_rows_plain(const VerifyParams p) {
     }
 }
 
-constexpr int kFinishThreads = 256;
+constexpr int kFinishThreads = 1024;   // one sweep for drafts of up to 1024 tokens
 
 template <typename T>
 __global__ void __launch_bounds__(kFinishThreads) verify_finish_kernel(
@@ -392,13 +392,25 @@ __global__ void __launch_bounds__(kFinishThreads) verify_finish_kernel(
     int myfirst = K;
     for (int i = tid; i < K; i += blockDim.x) {
         const int64_t r = i0 + i;
+        // P (reference, sum) pairs of this row; read two at a time where P is even
         const float2 *pp = partials + r * P;
-        float Mx = kNegInit;
-        for (int q = 0; q < P; ++q) Mx = fmaxf(Mx, pp[q].x);
-        float S = 0.f;
-        for (int q = 0; q < P; ++q) {
-            const float2 v = pp[q];
-            S += v.y * expf(v.x - Mx);
+        float Mx = kNegInit, S = 0.f;
+        if ((P & 1) == 0) {
+            const float4 *p4 = reinterpret_cast<const float4 *>(pp);
+            for (int q = 0; q < P / 2; ++q) {
+                const float4 v = p4[q];
+                Mx = fmaxf(Mx, fmaxf(v.x, v.z));
+            }
+            for (int q = 0; q < P / 2; ++q) {
+                const float4 v = p4[q];
+                S += v.y * ex2((v.x - Mx) * kLog2e) + v.w * ex2((v.z - Mx) * kLog2e);
+            }
+        } else {
+            for (int q = 0; q < P; ++q) Mx = fmaxf(Mx, pp[q].x);
+            for (int q = 0; q < P; ++q) {
+                const float2 v = pp[q];
+                S += v.y * ex2((v.x - Mx) * kLog2e);
+            }
         }
         const float lse = Mx + logf(S);
         if (!(fabsf(lse) < INFINITY)) myflags |= SSD_UTT_NONFINITE;
