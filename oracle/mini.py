@@ -60,3 +60,24 @@ def accepted_prefix(likelihoods, tau_slm):
     """Section 2.3: j = min{i : p_i <= tau} (1-based); returns j-1, or len if no such i."""
     bad = [i for i, p in enumerate(likelihoods) if p <= tau_slm]
     return min(bad) if bad else len(likelihoods)
+
+
+def sweep(max_entropy, likelihoods, pairs):
+    """Section 3.2's operating-point sweep for one utterance: for every (tau_ctc, tau_slm)
+    pair, whether the gate passes and how long the verified prefix is."""
+    return [(max_entropy < tc, accepted_prefix(likelihoods, ts)) for tc, ts in pairs]
+
+
+def final_hypothesis(draft, gate_ok, likelihoods, tau_slm):
+    """Eq. 7 for one utterance: (tokens that are final so far, needs the AR pass?)."""
+    j = accepted_prefix(likelihoods, tau_slm)
+    if gate_ok or j == len(draft):
+        return list(draft), False
+    return list(draft[:j]), True
+
+
+def greedy_token(x):
+    """Eq. 6, one step: the most likely token (first maximiser) and its log-likelihood."""
+    logp, p = log_softmax(x)
+    v = int(np.argmax(p))
+    return v, float(logp[v])

@@ -22,7 +22,8 @@ def lib():
         _lib.ssd_ref_row_stats.restype = C.c_int
         _lib.ssd_ref_collapse.restype = C.c_int32
         for name in ("ssd_ref_ctc_draft", "ssd_ref_entropy_gate", "ssd_ref_verify",
-                     "ssd_ref_set_threads"):
+                     "ssd_ref_set_threads", "ssd_ref_threshold_sweep", "ssd_ref_assemble",
+                     "ssd_ref_greedy_step"):
             getattr(_lib, name).restype = C.c_int32
     return _lib
 
@@ -122,4 +123,58 @@ def verify(logits, V, tok_off, draft_ids, tau_slm, skip=None):
         _p(o["utt_status"]))
     if rc != 0:
         raise ValueError("ssd_ref_verify rejected its arguments (code %d)" % rc)
+    return o
+
+
+def threshold_sweep(utt_max_entropy, token_logp, tok_off, tau_ctc, tau_slm):
+    """Gate and first reject for every (tau_ctc[p], tau_slm[p]) pair (Section 3.2's sweep)."""
+    h = np.ascontiguousarray(utt_max_entropy, np.float64)
+    lp = np.ascontiguousarray(token_logp, np.float64)
+    tok_off = np.ascontiguousarray(tok_off, np.int64)
+    tc = np.ascontiguousarray(tau_ctc, np.float64)
+    ts = np.ascontiguousarray(tau_slm, np.float64)
+    B, M, P = tok_off.shape[0] - 1, lp.shape[0], tc.shape[0]
+    assert ts.shape[0] == P and h.shape[0] == B
+    o = dict(gate_accept=np.zeros((P, B), np.uint8), accepted_len=np.zeros((P, B), np.int32),
+             all_accepted=np.zeros((P, B), np.uint8), counts=np.zeros((P, 3), np.int32))
+    rc = lib().ssd_ref_threshold_sweep(_p(h), _p(lp), _p(tok_off), C.c_int32(B), C.c_int64(M),
+                                       _p(tc), _p(ts), C.c_int32(P), _p(o["gate_accept"]),
+                                       _p(o["accepted_len"]), _p(o["all_accepted"]), _p(o["counts"]))
+    if rc != 0:
+        raise ValueError("ssd_ref_threshold_sweep rejected its arguments (code %d)" % rc)
+    return o
+
+
+def assemble(tokens, tok_off, gate_accept, accepted_len, all_accepted):
+    """Eq. 7: final hypotheses and the list of utterances left to the AR pass."""
+    tokens = np.ascontiguousarray(tokens, np.int32)
+    tok_off = np.ascontiguousarray(tok_off, np.int64)
+    B, M = tok_off.shape[0] - 1, tokens.shape[0]
+    g = np.ascontiguousarray(gate_accept, np.uint8)
+    a = np.ascontiguousarray(accepted_len, np.int32)
+    aa = np.ascontiguousarray(all_accepted, np.uint8)
+    o = dict(final_tokens=np.full(M, -1, np.int32), final_len=np.zeros(B, np.int32),
+             is_final=np.zeros(B, np.uint8), ar_utt=np.full(B, -1, np.int32),
+             ar_resume=np.full(B, -1, np.int32))
+    n = C.c_int32(0)
+    rc = lib().ssd_ref_assemble(_p(tokens), _p(tok_off), C.c_int32(B), C.c_int64(M), _p(g), _p(a),
+                                _p(aa), _p(o["final_tokens"]), _p(o["final_len"]),
+                                _p(o["is_final"]), C.byref(n), _p(o["ar_utt"]), _p(o["ar_resume"]))
+    if rc != 0:
+        raise ValueError("ssd_ref_assemble rejected its arguments (code %d)" % rc)
+    o["ar_count"] = int(n.value)
+    return o
+
+
+def greedy_step(logits, V):
+    """One greedy decoding step (Eq. 6) per row: most likely token and its log-likelihood."""
+    logits = np.ascontiguousarray(logits)
+    R, ld = logits.shape
+    o = dict(next_token=np.zeros(R, np.int32), next_logp=np.zeros(R, np.float64),
+             row_lse=np.zeros(R, np.float64), row_bad=np.zeros(R, np.uint8))
+    rc = lib().ssd_ref_greedy_step(_p(logits), C.c_int32(_dtype_code(logits)), C.c_int32(V),
+                                   C.c_int64(ld), C.c_int64(R), _p(o["next_token"]),
+                                   _p(o["next_logp"]), _p(o["row_lse"]), _p(o["row_bad"]))
+    if rc != 0:
+        raise ValueError("ssd_ref_greedy_step rejected its arguments (code %d)" % rc)
     return o

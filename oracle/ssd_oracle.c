@@ -23,6 +23,15 @@
  * bits of an IEEE binary32); softmax is the two-pass definition (max, then sum of
  * exponentials); no blocking, fusion or reordering.
  *
+ *   threshold sweep  -- the operating-point study of Section 3.2 / Table 1: the gate of
+ *                       Eq. 3 and the first reject of Section 2.3 re-evaluated for a list
+ *                       of (tau_CTC, tau_SLM) pairs from stored per-utterance maxima and
+ *                       per-token log-likelihoods;
+ *   assemble         -- Eq. 7: the final hypothesis is the draft if Eq. 3 or Eq. 5 holds,
+ *                       else the verified prefix, to be continued by the AR pass;
+ *   greedy step      -- one step of Eq. 6's greedy decoding: the most likely next token
+ *                       under the LLM's softmax and its log-likelihood.
+ *
  * Parity pins (tests/test_oracle_pins.py): closed-form entropies (uniform, one-hot,
  * k-of-V, binary), planted probability vectors, shift invariance, brute-force
  * enumeration of alignments and of collapses on tiny vocabularies, planted reject
@@ -274,6 +283,111 @@ int32_t ssd_ref_verify(const void *logits, int32_t dtype, int32_t V, int64_t ld,
         accepted_len[b] = first_reject;
         all_accepted[b] = (uint8_t)(first_reject == K);
         if (utt_status) utt_status[b] = st;
+    }
+    return 0;
+}
+
+/*
+ * Operating points from one pass (Section 3.2 sweeps tau_CTC in [0.7, 3.0] with
+ * tau_SLM in {0.1, 0.2}).  For pair p and utterance b:
+ *   gate_accept[p*B+b]  = (utt_max_entropy[b] < tau_ctc[p])            (Eq. 3: max over frames)
+ *   accepted_len[p*B+b] = first i with exp(token_logp[i]) <= tau_slm[p], else K_b  (Section 2.3)
+ *   all_accepted[p*B+b] = (accepted_len == K_b)                                     (Eq. 5)
+ * counts (nullable) [P,3]: utterances final by the gate / final by verification only /
+ * left to the AR pass.  A NaN maximum never passes; a NaN likelihood is a reject;
+ * tau_slm <= 0 rejects nothing.  Malformed offsets: accepted_len 0, all_accepted 0.
+ */
+int32_t ssd_ref_threshold_sweep(const double *utt_max_entropy, const double *token_logp,
+                                const int64_t *tok_off, int32_t B, int64_t M,
+                                const double *tau_ctc, const double *tau_slm, int32_t P,
+                                uint8_t *gate_accept, int32_t *accepted_len,
+                                uint8_t *all_accepted, int32_t *counts) {
+    if (B < 0 || M < 0 || P < 0) return 2;
+    for (int32_t p = 0; p < P; ++p) {
+        int32_t n_gate = 0, n_verify = 0, n_ar = 0;
+        for (int32_t b = 0; b < B; ++b) {
+            int64_t o = (int64_t)p * B + b;
+            int g = utt_max_entropy[b] < tau_ctc[p];
+            int32_t K = 0, first = 0;
+            int all = 0;
+            if (offsets_ok(tok_off, b, M)) {
+                K = (int32_t)(tok_off[b + 1] - tok_off[b]);
+                first = K;
+                for (int32_t i = 0; i < K; ++i) {
+                    double prob = exp(token_logp[tok_off[b] + i]);
+                    int reject = !(prob > tau_slm[p]);
+                    if (tau_slm[p] <= 0.0) reject = 0;
+                    if (reject) { first = i; break; }
+                }
+                all = (first == K);
+            }
+            gate_accept[o] = (uint8_t)g;
+            accepted_len[o] = first;
+            all_accepted[o] = (uint8_t)all;
+            if (g) ++n_gate; else if (all) ++n_verify; else ++n_ar;
+        }
+        if (counts) { counts[3 * p] = n_gate; counts[3 * p + 1] = n_verify; counts[3 * p + 2] = n_ar; }
+    }
+    return 0;
+}
+
+/*
+ * Eq. 7.  tokens[tok_off[b] .. tok_off[b+1]) is the draft of utterance b in the token space it
+ * was verified in.  If the gate accepted it (Eq. 3) or every token passed (Eq. 5) the draft is
+ * final: final_len = K_b, is_final = 1.  Otherwise the final hypothesis starts with the
+ * verified prefix (accepted_len tokens, Section 2.3) and the utterance joins the list for the
+ * AR pass: ar_utt (ascending utterance ids), ar_resume (length of the prefix = position the AR
+ * pass generates first), *ar_count.  final_tokens has the layout of tokens; only the first
+ * final_len[b] entries of an utterance are written.
+ */
+int32_t ssd_ref_assemble(const int32_t *tokens, const int64_t *tok_off, int32_t B, int64_t M,
+                         const uint8_t *gate_accept, const int32_t *accepted_len,
+                         const uint8_t *all_accepted,
+                         int32_t *final_tokens, int32_t *final_len, uint8_t *is_final,
+                         int32_t *ar_count, int32_t *ar_utt, int32_t *ar_resume) {
+    if (B < 0 || M < 0) return 2;
+    int32_t n = 0;
+    for (int32_t b = 0; b < B; ++b) {
+        int32_t K = 0;
+        if (offsets_ok(tok_off, b, M)) K = (int32_t)(tok_off[b + 1] - tok_off[b]);
+        int fin = (gate_accept[b] != 0) || (all_accepted[b] != 0);
+        int32_t len = K;
+        if (!fin) {
+            len = accepted_len[b];
+            if (len < 0) len = 0;
+            if (len > K) len = K;
+        }
+        for (int32_t i = 0; i < len; ++i) final_tokens[tok_off[b] + i] = tokens[tok_off[b] + i];
+        final_len[b] = len;
+        is_final[b] = (uint8_t)fin;
+        if (!fin) { ar_utt[n] = b; ar_resume[n] = len; ++n; }
+    }
+    *ar_count = n;
+    return 0;
+}
+
+/*
+ * One greedy step of Eq. 6 for R independent rows of LLM logits [R, ld]:
+ *   next_token[r] = argmax_v p(v | ...) = smallest v attaining the largest logit
+ *   next_logp[r]  = log p(next_token[r] | ...) = x_max - lse            (nullable)
+ *   row_lse[r]                                                          (nullable)
+ * Returns the number of rows whose lse is not finite in *bad_rows (nullable).
+ */
+int32_t ssd_ref_greedy_step(const void *logits, int32_t dtype, int32_t V, int64_t ld, int64_t R,
+                            int32_t *next_token, double *next_logp, double *row_lse,
+                            uint8_t *row_bad) {
+    if (!logits && R > 0) return 1;
+    if (V < 1 || ld < V || R < 0) return 2;
+    if (dtype != SSD_REF_F32 && dtype != SSD_REF_BF16) return 3;
+#pragma omp parallel for schedule(dynamic, 16)
+    for (int64_t r = 0; r < R; ++r) {
+        double l;
+        int32_t arg;
+        int ok = ssd_ref_row_stats(logits, dtype, r * ld, V, &l, NULL, &arg, NULL);
+        next_token[r] = arg;
+        if (next_logp) next_logp[r] = ref_load(logits, dtype, r * ld + arg) - l;
+        if (row_lse) row_lse[r] = l;
+        if (row_bad) row_bad[r] = (uint8_t)!ok;
     }
     return 0;
 }

@@ -47,8 +47,46 @@ class COracle:
         return o["token_logp"], int(o["accepted_len"][0]), bool(o["all_accepted"][0])
 
 
+    def sweep(self, max_entropy, logp, pairs):
+        K = len(logp)
+        o = ref.threshold_sweep([max_entropy], np.asarray(logp, np.float64), [0, K],
+                                [p[0] for p in pairs], [p[1] for p in pairs])
+        for i in range(len(pairs)):
+            assert o["counts"][i].sum() == 1
+            assert bool(o["all_accepted"][i, 0]) == (o["accepted_len"][i, 0] == K)
+        return [(bool(o["gate_accept"][i, 0]), int(o["accepted_len"][i, 0]))
+                for i in range(len(pairs))]
+
+    def assemble(self, draft, gate_ok, logp, tau):
+        K = len(draft)
+        sw = ref.threshold_sweep([0.0], np.asarray(logp, np.float64), [0, K], [1.0], [tau])
+        o = ref.assemble(np.asarray(draft, np.int32), [0, K], [1 if gate_ok else 0],
+                         sw["accepted_len"][0], sw["all_accepted"][0])
+        n = int(o["final_len"][0])
+        needs_ar = o["ar_count"] == 1
+        assert needs_ar == (not o["is_final"][0])
+        if needs_ar:
+            assert o["ar_utt"][0] == 0 and o["ar_resume"][0] == n
+        return [int(v) for v in o["final_tokens"][:n]], bool(needs_ar)
+
+    def greedy(self, x):
+        x = np.ascontiguousarray(x)
+        o = ref.greedy_step(x.reshape(1, -1), x.shape[0])
+        return int(o["next_token"][0]), float(o["next_logp"][0])
+
+
 class MiniOracle:
     name = "numpy-mini-oracle"
+
+    def sweep(self, max_entropy, logp, pairs):
+        with np.errstate(over="ignore"):
+            return [(bool(g), int(n)) for g, n in mini.sweep(max_entropy, np.exp(np.asarray(logp, np.float64)), pairs)]
+
+    def assemble(self, draft, gate_ok, logp, tau):
+        return mini.final_hypothesis(draft, gate_ok, np.exp(np.asarray(logp, np.float64)), tau)
+
+    def greedy(self, x):
+        return mini.greedy_token(mini.widen(x))
 
     def row(self, x):
         x = mini.widen(x)
@@ -249,9 +287,89 @@ class VerifyShiftedRow(_Mutant):
             return np.log(np.array(p)), n, n == K
 
 
+class SweepNonStrictGate(_Mutant):
+    name = "mutant: sweep gate uses <="
+
+    def sweep(self, max_entropy, logp, pairs):
+        return [(max_entropy <= tc, n) for (tc, _), (_, n) in zip(pairs, super().sweep(max_entropy, logp, pairs))]
+
+
+class SweepIgnoresPairIndex(_Mutant):
+    name = "mutant: sweep evaluates every pair with the first pair's thresholds"
+
+    def sweep(self, max_entropy, logp, pairs):
+        return super().sweep(max_entropy, logp, [pairs[0]] * len(pairs))
+
+
+class SweepComparesLogpWithTau(_Mutant):
+    name = "mutant: sweep compares the log-likelihood with tau itself"
+
+    def sweep(self, max_entropy, logp, pairs):
+        out = []
+        for tc, ts in pairs:
+            bad = [i for i, lp in enumerate(logp) if lp <= ts]
+            out.append((max_entropy < tc, min(bad) if bad else len(logp)))
+        return out
+
+
+class AssembleKeepsRejectedToken(_Mutant):
+    name = "mutant: assembled prefix includes the rejected token"
+
+    def assemble(self, draft, gate_ok, logp, tau):
+        toks, ar = super().assemble(draft, gate_ok, logp, tau)
+        return (list(draft[:len(toks) + 1]), ar) if ar else (toks, ar)
+
+
+class AssembleIgnoresGate(_Mutant):
+    name = "mutant: a gate-accepted draft that fails verification is sent to the AR pass"
+
+    def assemble(self, draft, gate_ok, logp, tau):
+        return super().assemble(draft, False, logp, tau)
+
+
+class AssembleRequiresBoth(_Mutant):
+    name = "mutant: final only if gate AND verification hold"
+
+    def assemble(self, draft, gate_ok, logp, tau):
+        toks, ar = super().assemble(draft, False, logp, tau)
+        if not gate_ok and not ar:
+            return toks, True
+        return toks, ar
+
+
+class GreedyArgmin(_Mutant):
+    name = "mutant: greedy step takes the least likely token"
+
+    def greedy(self, x):
+        xx = mini.widen(x)
+        logp, _ = mini.log_softmax(xx)
+        v = int(np.argmin(xx))
+        return v, float(logp[v])
+
+
+class GreedyUnnormalised(_Mutant):
+    name = "mutant: greedy step returns the raw logit as log-likelihood"
+
+    def greedy(self, x):
+        xx = mini.widen(x)
+        v = int(np.argmax(xx))
+        return v, float(xx[v])
+
+
+class GreedyLastOnTies(_Mutant):
+    name = "mutant: greedy step returns the last maximiser"
+
+    def greedy(self, x):
+        xx = mini.widen(x)
+        v = int(len(xx) - 1 - np.argmax(xx[::-1]))
+        return v, mini.greedy_token(xx)[1]
+
+
 ORACLES = [COracle(), MiniOracle()]
 MUTANTS = [EntropyWrongSign(), EntropyBase2(), EntropyDropsLseTerm(), LseWithoutMax(),
            ArgmaxLastOnTies(), ArgminInsteadOfArgmax(), CollapseBlanksFirst(),
            CollapseKeepsBlanks(), CollapseNoMerge(), GateNonStrict(), GateMean(), GateAny(),
            VerifyStrictReject(), VerifyOneBased(), VerifyLastReject(), VerifyTransposedGather(),
-           VerifyShiftedRow()]
+           VerifyShiftedRow(), SweepNonStrictGate(), SweepIgnoresPairIndex(),
+           SweepComparesLogpWithTau(), AssembleKeepsRejectedToken(), AssembleIgnoresGate(),
+           AssembleRequiresBoth(), GreedyArgmin(), GreedyUnnormalised(), GreedyLastOnTies()]

@@ -284,4 +284,76 @@ def pin_verify_rows_and_columns(impl):
     assert n == 2 and ok is False
 
 
+# ---- operating points from one pass (Section 3.2, Table 1 caption) ---------------------------
+
+def pin_sweep_planted(impl):
+    """Likelihoods worked by hand: for each tau_SLM the first position with p <= tau."""
+    q = [0.9, 0.5, 0.3, 0.15, 0.6, 0.05]
+    logp = [math.log(v) for v in q]
+    by_tau = {0.0: 6, 0.01: 6, 0.06: 5, 0.1: 5, 0.16: 3, 0.2: 3, 0.31: 2, 0.4: 2, 0.51: 1, 0.7: 1,
+              0.91: 0, 0.95: 0}      # thresholds sit strictly between the likelihoods
+    h = 1.2
+    gates = {0.7: False, 1.2: False, math.nextafter(1.2, 2): True, 3.0: True}
+    pairs = [(tc, ts) for tc in gates for ts in by_tau]
+    got = impl.sweep(h, logp, pairs)
+    assert len(got) == len(pairs)
+    for (tc, ts), (g, n) in zip(pairs, got):
+        assert g is gates[tc] and n == by_tau[ts], (tc, ts, g, n)
+    # the paper's two operating points on this utterance
+    assert impl.sweep(h, logp, [(0.7, 0.2), (3.0, 0.1)]) == [(False, 3), (True, 5)]
+
+
+def pin_sweep_monotone_and_empty(impl):
+    rng = np.random.default_rng(5)
+    logp = np.log(rng.uniform(0.02, 0.98, size=40)).tolist()
+    taus = sorted(rng.uniform(0, 1, size=25).tolist())
+    got = impl.sweep(0.5, logp, [(t * 3, t) for t in taus])
+    lens = [n for _, n in got]
+    assert all(a >= b for a, b in zip(lens, lens[1:]))       # a larger tau_SLM rejects earlier
+    gates = [g for g, _ in got]
+    assert gates == sorted(gates)                            # a larger tau_CTC accepts more
+    for t, (_, n) in zip(taus, got):                         # definition, position by position
+        assert all(math.exp(v) > t for v in logp[:n]) and (n == 40 or math.exp(logp[n]) <= t)
+    assert impl.sweep(0.0, [], [(0.0, 0.5), (0.1, 0.5)]) == [(False, 0), (True, 0)]
+
+
+# ---- Eq. 7 -----------------------------------------------------------------------------------
+
+def pin_assemble_cases(impl):
+    draft = [7, 8, 9, 10]
+    ok = [math.log(0.8)] * 4
+    bad2 = [math.log(0.8), math.log(0.7), math.log(0.01), math.log(0.9)]
+    bad0 = [math.log(0.05)] + ok[1:]
+    assert impl.assemble(draft, True, bad2, 0.1) == (draft, False)      # Eq. 3 holds
+    assert impl.assemble(draft, False, ok, 0.1) == (draft, False)       # Eq. 5 holds
+    assert impl.assemble(draft, True, ok, 0.1) == (draft, False)
+    assert impl.assemble(draft, False, bad2, 0.1) == ([7, 8], True)     # prefix before j
+    assert impl.assemble(draft, False, bad0, 0.1) == ([], True)
+    assert impl.assemble([], False, [], 0.1) == ([], False)             # vacuous Eq. 5
+    last = ok[:3] + [math.log(0.0999)]                                  # only the last token fails
+    assert impl.assemble(draft, False, last, 0.1) == ([7, 8, 9], True)
+
+
+# ---- Eq. 6, one step -------------------------------------------------------------------------
+
+def pin_greedy_planted(impl):
+    rng = np.random.default_rng(9)
+    for V in (1, 2, 17, 300):
+        q = rng.dirichlet(np.ones(V))
+        x = to_storage(np.log(q) + 2.5, "f32")
+        v, lp = impl.greedy(x)
+        assert v == int(np.argmax(q))
+        _close(lp, math.log(q.max()), 1e-6, "greedy logp V=%d" % V)
+    x = np.zeros(9, np.float32)
+    x[[2, 5, 7]] = 4.0                                      # three equal maxima
+    v, lp = impl.greedy(x)
+    assert v == 2
+    _close(lp, 4.0 - math.log(3 * math.exp(4.0) + 6), 1e-12, "tie logp")
+    v, lp = impl.greedy(np.array([3.25], np.float32))
+    assert v == 0 and abs(lp) < 1e-15
+    v, lp = impl.greedy(to_storage(np.array([-1.0, 2.0, 0.5]), "bf16"))
+    assert v == 1
+    _close(lp, 2.0 - math.log(math.exp(-1.0) + math.exp(2.0) + math.exp(0.5)), 1e-12, "bf16 row")
+
+
 ALL_PINS = [v for k, v in sorted(globals().items()) if k.startswith("pin_")]
