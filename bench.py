@@ -291,6 +291,7 @@ def run_ours(args):
     if rank != 0:
         D.finalize()
         return
+    next_rows = None if args.ncu_small else time_next_rows(sets, device, peak)
     s0 = sets[0]
     gate_acc = float(s0["gate"]["gate_accept"].float().mean().item())
     all_acc = s0["s2"]["all_accepted"].cpu().numpy().astype(bool)
@@ -322,11 +323,74 @@ def run_ours(args):
                           round(float(all_acc[~skipped].mean()) if (~skipped).any() else 0.0, 4)},
         "clocks": summarise_clocks(clock_rows, windows, clock_note),
         "e2e": e2e,
+        "next_rows": next_rows,
     }
     if world == 1 and not args.no_cpu_baseline and not args.ncu_small:
         line["cpu_baseline"] = cpu_baseline(s0, budget_s=12.0)
     print(json.dumps(line), flush=True)
     D.finalize()
+
+
+def time_next_rows(sets, device, peak):
+    """The calls that follow the path (not part of `value`): the operating-point sweep over the
+    step's stored maxima and log-likelihoods, the assembly of Eq. 7, and one greedy decoding
+    step over as many rows as the step has utterances left to the auto-regressive pass would
+    be too small to time, so over the first 1024 verify rows of each input set in turn."""
+    import torch
+    from paper_2603_11243_b200 import binding as ssd
+    n_sets = len(sets)
+    pairs = [(0.7 + 2.3 * i / 15.0, ts) for i in range(16) for ts in (0.1, 0.2)]
+    tc, ts = [p[0] for p in pairs], [p[1] for p in pairs]
+    R = min(1024, min(s["M"] for s in sets))
+    prep = []
+    for s in sets:
+        sw = ssd.ssd_threshold_sweep(s["s1"]["utt_max_entropy"], s["s2"]["token_logp"],
+                                     s["tok_off"], tc, ts)
+        asm = ssd.ssd_assemble(s["ids"], s["tok_off"], s["gate"]["gate_accept"],
+                               s["s2"]["accepted_len"], s["s2"]["all_accepted"])
+        gr = ssd.ssd_greedy_step(s["vb"].logits[:R])
+        prep.append((sw, asm, gr))
+    torch.cuda.synchronize()
+
+    def timed(fn, n=60):
+        for i in range(6):
+            fn(i % n_sets)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for i in range(n):
+            fn(i % n_sets)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n * 1e3
+
+    t_sw = timed(lambda i: ssd.ssd_threshold_sweep(
+        sets[i]["s1"]["utt_max_entropy"], sets[i]["s2"]["token_logp"], sets[i]["tok_off"], tc, ts,
+        out=prep[i][0]))
+    t_asm = timed(lambda i: ssd.ssd_assemble(
+        sets[i]["ids"], sets[i]["tok_off"], sets[i]["gate"]["gate_accept"],
+        sets[i]["s2"]["accepted_len"], sets[i]["s2"]["all_accepted"], out=prep[i][1]))
+    t_gr = timed(lambda i: ssd.ssd_greedy_step(sets[i]["vb"].logits[:R], out=prep[i][2]))
+    # the streaming kernel alone, from events the library records around it
+    kev = make_events(2 * 12)
+    for j in range(12):
+        o = ssd.LaunchOpts()
+        o.ev_begin, o.ev_end = kev[2 * j].cuda_event, kev[2 * j + 1].cuda_event
+        ssd.ssd_greedy_step(sets[j % n_sets]["vb"].logits[:R], out=prep[j % n_sets][2], opts=o)
+    torch.cuda.synchronize()
+    t_gk = statistics.mean(kev[2 * j].elapsed_time(kev[2 * j + 1]) for j in range(2, 12)) * 1e3
+    w = sets[0]["w"]
+    gbytes = R * w.V_llm * (2 if w.dtype == "bf16" else 4)
+    return {"threshold_sweep": {"pairs": len(pairs), "us_per_call": round(t_sw, 2)},
+            "assemble": {"us_per_call": round(t_asm, 2),
+                         "ar_count": int(prep[0][1]["ar_count"].cpu()[0])},
+            "greedy_step": {"rows": R, "V": w.V_llm, "us_per_call": round(t_gr, 2),
+                            "kernel_us": round(t_gk, 2),
+                            "kernel_gbs": round(gbytes / (t_gk * 1e-6) / 1e9, 1),
+                            "kernel_frac": round(gbytes / (t_gk * 1e-6) / 1e9 / peak, 4),
+                            "note": "us_per_call is host-paced (Python marshalling included); "
+                                    "kernel_* is the streaming kernel between two events; rows "
+                                    "from %d input sets in turn" % n_sets}}
 
 
 def run_e2e(s, device, steps, D, world):

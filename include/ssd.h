@@ -179,6 +179,76 @@ int32_t ssd_verify(const void *logits, ssd_dtype dtype, int32_t V, int64_t ld,
                    const ssd_launch_opts *opts);
 
 /*
+ * Operating points from one pass.  Section 3.2 of the paper studies tau_CTC in [0.7, 3.0] and
+ * tau_SLM in {0.1, 0.2} (Table 1 gives two of the points); both decisions depend on the logits
+ * only through the per-utterance maximum entropy (Eq. 3) and the per-token log-likelihoods
+ * (Eq. 5), which ssd_ctc_draft / ssd_entropy_gate and ssd_verify leave behind.  For every pair
+ * p < P and utterance b:
+ *   gate_accept[p*B + b]  = (utt_max_entropy[b] < tau_ctc[p])            (Eq. 3; NaN never passes)
+ *   accepted_len[p*B + b] = first i with token_logp[i] <= log(tau_slm[p]), else K_b   (Section 2.3)
+ *   all_accepted[p*B + b] = (accepted_len == K_b)                                     (Eq. 5)
+ *   counts[3*p + 0..2]    = utterances final by the gate / final by verification only / left
+ *                           to the auto-regressive pass                                (nullable)
+ * tau_slm[p] <= 0 rejects nothing; a NaN or -inf log-likelihood is a reject otherwise.  The
+ * verification outcome is computed for every utterance, gate-accepted or not (token_logp of
+ * utterances ssd_verify skipped is whatever the caller left there).  Malformed offsets give
+ * accepted_len 0, all_accepted 0.
+ * utt_max_entropy [B] f32, token_logp [M] f32, tok_off [B+1] int64: device.
+ * tau_ctc, tau_slm [P] f32: HOST arrays, read during the call.
+ * gate_accept, all_accepted [P*B] u8, accepted_len [P*B] i32, counts [P*3] i32: device.
+ * Errors: SSD_ERR_NULL, SSD_ERR_ARG, SSD_ERR_CUDA.
+ */
+int32_t ssd_threshold_sweep(const float *utt_max_entropy, const float *token_logp,
+                            const int64_t *tok_off, int32_t B, int64_t M,
+                            const float *tau_ctc, const float *tau_slm, int32_t P,
+                            uint8_t *gate_accept, int32_t *accepted_len, uint8_t *all_accepted,
+                            int32_t *counts, void *stream);
+
+/*
+ * The final hypothesis, Eq. 7 of the paper, and the hand-over to the auto-regressive pass
+ * (Section 2.3; Section 3.2 batches that pass separately).  tokens[tok_off[b] .. tok_off[b+1])
+ * is the draft of utterance b in the token space it was verified in.  If Eq. 3 or Eq. 5 holds
+ * (gate_accept[b] or all_accepted[b] nonzero) the draft is final; otherwise the hypothesis
+ * starts with the verified prefix of accepted_len[b] tokens and the utterance is listed for
+ * the auto-regressive pass:
+ *   final_tokens  same layout as tokens; the first final_len[b] entries of an utterance are
+ *                 written, the rest left untouched
+ *   final_len[b]  K_b if final, else accepted_len[b] clamped to [0, K_b]
+ *   is_final[b]   1 / 0
+ *   ar_count[0]   number of utterances that are not final
+ *   ar_utt[k], ar_resume[k], k < ar_count: their ids in ascending order and the length of
+ *                 their verified prefix (the position the auto-regressive pass generates first)
+ * All pointers device.  tokens, final_tokens [M] i32; final_len, ar_utt, ar_resume [B] i32;
+ * is_final [B] u8; ar_count [1] i32.
+ * Errors: SSD_ERR_NULL, SSD_ERR_ARG, SSD_ERR_CUDA.
+ */
+int32_t ssd_assemble(const int32_t *tokens, const int64_t *tok_off, int32_t B, int64_t M,
+                     const uint8_t *gate_accept, const int32_t *accepted_len,
+                     const uint8_t *all_accepted,
+                     int32_t *final_tokens, int32_t *final_len, uint8_t *is_final,
+                     int32_t *ar_count, int32_t *ar_utt, int32_t *ar_resume, void *stream);
+
+/*
+ * One step of the greedy auto-regressive fallback, Eq. 6 of the paper: for each of R rows of
+ * LLM logits (one row per utterance still decoding),
+ *   next_token[r] = argmax_v p(v | ...)   (lowest index on ties)
+ *   next_logp[r]  = log p(next_token[r] | ...) = x[r, next_token[r]] - row_lse[r]   (nullable)
+ *   row_lse[r]    = log sum_v exp(x[r, v])                                           (nullable)
+ *   row_status[r] = SSD_UTT_NONFINITE for a row holding NaN / +inf or only -inf      (nullable)
+ * logits [R, ld] dtype, read once by the same streaming kernel as ssd_verify, which here also
+ * tracks the running maximum and its first position.
+ * workspace: at least ssd_greedy_step_workspace_bytes(...) bytes, 256-byte aligned.
+ * Errors: SSD_ERR_NULL, SSD_ERR_ARG (also opts->kernel == 1: the plain-load kernel has no
+ * arg-max variant), SSD_ERR_DTYPE, SSD_ERR_ALIGN, SSD_ERR_WORKSPACE, SSD_ERR_CUDA.
+ */
+size_t ssd_greedy_step_workspace_bytes(int64_t R, int32_t V, ssd_dtype dtype,
+                                       const ssd_launch_opts *opts);
+int32_t ssd_greedy_step(const void *logits, ssd_dtype dtype, int32_t V, int64_t ld, int64_t R,
+                        int32_t *next_token, float *next_logp, float *row_lse,
+                        uint32_t *row_status, void *workspace, size_t workspace_bytes,
+                        void *stream, const ssd_launch_opts *opts);
+
+/*
  * ssd_verify without a workspace argument, for callers that cannot allocate device memory.
  * (The paper has no counterpart: this is a packaging variant of ssd_verify, same arithmetic.)
  *

@@ -67,6 +67,15 @@ def lib():
         L.ssd_verify_static.restype = i32
         L.ssd_verify_static.argtypes = [vp, C.c_int, i32, i64, vp, vp, i32, i64, C.c_float, vp,
                                         vp, vp, vp, vp, vp, vp, vp]
+        L.ssd_threshold_sweep.restype = i32
+        L.ssd_threshold_sweep.argtypes = [vp, vp, vp, i32, i64, vp, vp, i32, vp, vp, vp, vp, vp]
+        L.ssd_assemble.restype = i32
+        L.ssd_assemble.argtypes = [vp, vp, i32, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.ssd_greedy_step_workspace_bytes.restype = C.c_size_t
+        L.ssd_greedy_step_workspace_bytes.argtypes = [i64, i32, C.c_int, vp]
+        L.ssd_greedy_step.restype = i32
+        L.ssd_greedy_step.argtypes = [vp, C.c_int, i32, i64, i64, vp, vp, vp, vp, vp, C.c_size_t,
+                                      vp, vp]
         _lib = L
     return _lib
 
@@ -230,6 +239,94 @@ def ssd_verify_static(logits: torch.Tensor, tok_off: torch.Tensor, draft_ids: to
         _dev(out["utt_status"], "utt_status"), _stream(), _opts(opts))
     if rc != OK:
         raise SsdError(rc, "ssd_verify_static")
+    return out
+
+
+def ssd_threshold_sweep(utt_max_entropy: torch.Tensor, token_logp: torch.Tensor,
+                        tok_off: torch.Tensor, tau_ctc, tau_slm, out=None,
+                        want_counts: bool = True) -> Dict[str, torch.Tensor]:
+    """Gate and first reject for every (tau_ctc[p], tau_slm[p]) pair from stored maxima and
+    log-likelihoods (Section 3.2's operating-point sweep).  tau_ctc / tau_slm: host sequences."""
+    B, M = tok_off.shape[0] - 1, token_logp.shape[0]
+    P = len(tau_ctc)
+    if len(tau_slm) != P:
+        raise ValueError("tau_ctc and tau_slm must have the same length")
+    if utt_max_entropy.dtype != torch.float32 or token_logp.dtype != torch.float32:
+        raise TypeError("utt_max_entropy and token_logp must be float32")
+    if tok_off.dtype != torch.int64:
+        raise TypeError("tok_off must be int64")
+    dev = token_logp.device if M else utt_max_entropy.device
+    if out is None:
+        out = dict(gate_accept=torch.empty((P, B), dtype=torch.uint8, device=dev),
+                   accepted_len=torch.empty((P, B), dtype=torch.int32, device=dev),
+                   all_accepted=torch.empty((P, B), dtype=torch.uint8, device=dev))
+        if want_counts:
+            out["counts"] = torch.empty((P, 3), dtype=torch.int32, device=dev)
+    tc = (C.c_float * max(P, 1))(*[float(v) for v in tau_ctc])
+    ts = (C.c_float * max(P, 1))(*[float(v) for v in tau_slm])
+    rc = lib().ssd_threshold_sweep(
+        _dev(utt_max_entropy, "utt_max_entropy"), _dev(token_logp, "token_logp"),
+        _dev(tok_off, "tok_off"), B, M, C.cast(tc, C.c_void_p), C.cast(ts, C.c_void_p), P,
+        _dev(out["gate_accept"], "gate_accept"), _dev(out["accepted_len"], "accepted_len"),
+        _dev(out["all_accepted"], "all_accepted"), _dev(out.get("counts"), "counts"), _stream())
+    if rc != OK:
+        raise SsdError(rc, "ssd_threshold_sweep")
+    return out
+
+
+def ssd_assemble(tokens: torch.Tensor, tok_off: torch.Tensor, gate_accept: torch.Tensor,
+                 accepted_len: torch.Tensor, all_accepted: torch.Tensor,
+                 out=None) -> Dict[str, torch.Tensor]:
+    """Eq. 7: final hypotheses and the ordered list of utterances left to the AR pass."""
+    B, M = tok_off.shape[0] - 1, tokens.shape[0]
+    if tokens.dtype != torch.int32 or accepted_len.dtype != torch.int32:
+        raise TypeError("tokens and accepted_len must be int32")
+    if gate_accept.dtype != torch.uint8 or all_accepted.dtype != torch.uint8:
+        raise TypeError("gate_accept and all_accepted must be uint8")
+    if tok_off.dtype != torch.int64:
+        raise TypeError("tok_off must be int64")
+    dev = tok_off.device
+    if out is None:
+        e = lambda n, dt: torch.empty((n,), dtype=dt, device=dev)
+        out = dict(final_tokens=e(M, torch.int32), final_len=e(B, torch.int32),
+                   is_final=e(B, torch.uint8), ar_count=e(1, torch.int32),
+                   ar_utt=e(B, torch.int32), ar_resume=e(B, torch.int32))
+    rc = lib().ssd_assemble(
+        _dev(tokens, "tokens"), _dev(tok_off, "tok_off"), B, M, _dev(gate_accept, "gate_accept"),
+        _dev(accepted_len, "accepted_len"), _dev(all_accepted, "all_accepted"),
+        _dev(out["final_tokens"], "final_tokens"), _dev(out["final_len"], "final_len"),
+        _dev(out["is_final"], "is_final"), _dev(out["ar_count"], "ar_count"),
+        _dev(out["ar_utt"], "ar_utt"), _dev(out["ar_resume"], "ar_resume"), _stream())
+    if rc != OK:
+        raise SsdError(rc, "ssd_assemble")
+    return out
+
+
+def ssd_greedy_step_workspace_bytes(R, V, dtype_code, opts=None) -> int:
+    return int(lib().ssd_greedy_step_workspace_bytes(R, V, dtype_code, _opts(opts)))
+
+
+def ssd_greedy_step(logits: torch.Tensor, V: Optional[int] = None, out=None,
+                    opts: Optional[LaunchOpts] = None) -> Dict[str, torch.Tensor]:
+    """One greedy decoding step (Eq. 6) per row: most likely token and its log-likelihood."""
+    R, ld = _rows_ld(logits)
+    V = logits.shape[1] if V is None else V
+    code = _dtype_code(logits)
+    if out is None:
+        dev = logits.device
+        e = lambda n, dt: torch.empty((n,), dtype=dt, device=dev)
+        out = dict(next_token=e(R, torch.int32), next_logp=e(R, torch.float32),
+                   row_lse=e(R, torch.float32), row_status=e(R, torch.int32),
+                   workspace=torch.empty((max(ssd_greedy_step_workspace_bytes(R, V, code, opts), 256),),
+                                         dtype=torch.uint8, device=dev))
+    ws = out["workspace"]
+    rc = lib().ssd_greedy_step(
+        _dev(logits, "logits"), code, V, ld, R, _dev(out["next_token"], "next_token"),
+        _dev(out.get("next_logp"), "next_logp"), _dev(out.get("row_lse"), "row_lse"),
+        _dev(out.get("row_status"), "row_status"), _dev(ws, "workspace"), ws.numel(), _stream(),
+        _opts(opts))
+    if rc != OK:
+        raise SsdError(rc, "ssd_greedy_step")
     return out
 
 

@@ -110,4 +110,65 @@ int32_t ssd_verify(const void *logits, ssd_dtype dtype, int32_t V, int64_t ld,
                          token_logp, row_lse, accepted_len, all_accepted, utt_status, plan, L);
 }
 
+int32_t ssd_threshold_sweep(const float *utt_max_entropy, const float *token_logp,
+                            const int64_t *tok_off, int32_t B, int64_t M,
+                            const float *tau_ctc, const float *tau_slm, int32_t P,
+                            uint8_t *gate_accept, int32_t *accepted_len, uint8_t *all_accepted,
+                            int32_t *counts, void *stream) {
+    if (B < 0 || M < 0 || P < 0) return SSD_ERR_ARG;
+    if (!tok_off) return SSD_ERR_NULL;
+    if (P > 0 && (!tau_ctc || !tau_slm)) return SSD_ERR_NULL;
+    if (P > 0 && B > 0 && (!utt_max_entropy || !gate_accept || !accepted_len || !all_accepted))
+        return SSD_ERR_NULL;
+    if (M > 0 && !token_logp) return SSD_ERR_NULL;
+    return launch_sweep(utt_max_entropy, token_logp, tok_off, B, M, tau_ctc, tau_slm, P,
+                        gate_accept, accepted_len, all_accepted, counts,
+                        static_cast<cudaStream_t>(stream));
+}
+
+int32_t ssd_assemble(const int32_t *tokens, const int64_t *tok_off, int32_t B, int64_t M,
+                     const uint8_t *gate_accept, const int32_t *accepted_len,
+                     const uint8_t *all_accepted,
+                     int32_t *final_tokens, int32_t *final_len, uint8_t *is_final,
+                     int32_t *ar_count, int32_t *ar_utt, int32_t *ar_resume, void *stream) {
+    if (B < 0 || M < 0) return SSD_ERR_ARG;
+    if (!tok_off || !ar_count) return SSD_ERR_NULL;
+    if (M > 0 && (!tokens || !final_tokens)) return SSD_ERR_NULL;
+    if (B > 0 && (!gate_accept || !accepted_len || !all_accepted || !final_len || !is_final ||
+                  !ar_utt || !ar_resume))
+        return SSD_ERR_NULL;
+    return launch_assemble(tokens, tok_off, B, M, gate_accept, accepted_len, all_accepted,
+                           final_tokens, final_len, is_final, ar_count, ar_utt, ar_resume,
+                           static_cast<cudaStream_t>(stream));
+}
+
+size_t ssd_greedy_step_workspace_bytes(int64_t R, int32_t V, ssd_dtype dtype,
+                                       const ssd_launch_opts *opts) {
+    if (R < 0 || V < 1 || (dtype != SSD_F32 && dtype != SSD_BF16)) return 0;
+    VerifyPlan plan;
+    if (plan_verify(0, R, V, dtype, opts, &plan) != SSD_OK) return 0;
+    return greedy_workspace_bytes(R, plan);
+}
+
+int32_t ssd_greedy_step(const void *logits, ssd_dtype dtype, int32_t V, int64_t ld, int64_t R,
+                        int32_t *next_token, float *next_logp, float *row_lse,
+                        uint32_t *row_status, void *workspace, size_t workspace_bytes,
+                        void *stream, const ssd_launch_opts *opts) {
+    if (dtype != SSD_F32 && dtype != SSD_BF16) return SSD_ERR_DTYPE;
+    if (R < 0 || V < 1 || ld < V) return SSD_ERR_ARG;
+    if (R > 0 && (!logits || !next_token)) return SSD_ERR_NULL;
+    const int es = dtype == SSD_F32 ? 4 : 2;
+    if (reinterpret_cast<uintptr_t>(logits) % es) return SSD_ERR_ALIGN;
+    VerifyPlan plan;
+    int rc = plan_verify(0, R, V, dtype, opts, &plan);
+    if (rc != SSD_OK) return rc;
+    if (plan.kernel != 2) return SSD_ERR_ARG;
+    if (R > 0 && (!workspace || workspace_bytes < greedy_workspace_bytes(R, plan) ||
+                  reinterpret_cast<uintptr_t>(workspace) % 256))
+        return SSD_ERR_WORKSPACE;
+    Launch L{static_cast<cudaStream_t>(stream), opts};
+    return launch_greedy(logits, dtype, V, ld, R, workspace, next_token, next_logp, row_lse,
+                         row_status, plan, L);
+}
+
 }  // extern "C"

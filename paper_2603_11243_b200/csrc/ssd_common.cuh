@@ -340,6 +340,21 @@ int launch_verify(const void *logits, ssd_dtype dtype, int V, int64_t ld, int64_
                   int32_t *accepted_len, uint8_t *all_accepted, uint32_t *utt_status,
                   const VerifyPlan &plan, const Launch &L);
 
+size_t greedy_workspace_bytes(int64_t R, const VerifyPlan &plan);
+int launch_greedy(const void *logits, ssd_dtype dtype, int V, int64_t ld, int64_t R,
+                  void *workspace, int32_t *next_token, float *next_logp, float *row_lse,
+                  uint32_t *row_status, const VerifyPlan &plan, const Launch &L);
+
+int launch_sweep(const float *utt_max_entropy, const float *token_logp, const int64_t *tok_off,
+                 int B, int64_t M, const float *tau_ctc, const float *tau_slm, int P,
+                 uint8_t *gate_accept, int32_t *accepted_len, uint8_t *all_accepted,
+                 int32_t *counts, cudaStream_t stream);
+int launch_assemble(const int32_t *tokens, const int64_t *tok_off, int B, int64_t M,
+                    const uint8_t *gate_accept, const int32_t *accepted_len,
+                    const uint8_t *all_accepted, int32_t *final_tokens, int32_t *final_len,
+                    uint8_t *is_final, int32_t *ar_count, int32_t *ar_utt, int32_t *ar_resume,
+                    cudaStream_t stream);
+
 void record_cuda_error(cudaError_t e);
 
 }  // namespace ssd

@@ -13,6 +13,7 @@
 //                      once per stage that the sum stayed in range (see Online), so the common
 //                      case is one exponential and no comparison per logit.
 //   verify_rows_plain  one CTA per item with scalar global loads; any alignment.  Fallback.
+#include <limits.h>
 #include <math.h>
 
 #include "ssd_common.cuh"
@@ -50,7 +51,31 @@ struct StageDesc {
     int32_t nchunks;
     uint32_t flags;
     int64_t slot;         // index of this item's first partial
+    int32_t elem0;        // row-relative index of the first element of the stage's first chunk
+    int32_t pad;
 };
+
+// Running arg max of one thread (the greedy-step variant): value and row-relative index of the
+// first element that attains it.
+struct ArgTrack {
+    float vmax;
+    int vidx;
+    __device__ __forceinline__ void reset() { vmax = -INFINITY; vidx = INT_MAX; }
+};
+template <typename T>
+__device__ __forceinline__ void track_chunk(const uint4 &w, int elem, ArgTrack &a) {
+    constexpr int EPC = Elem<T>::kPerChunk;
+    const float cm = chunk_max<T>(w);
+    if (cm > a.vmax) {                   // rare: a running maximum rises O(log n) times
+        float x[EPC];
+        chunk_unpack<T>(w, x);
+        int j = EPC - 1;
+#pragma unroll
+        for (int k = EPC - 2; k >= 0; --k) if (x[k] == cm) j = k;
+        a.vmax = cm;
+        a.vidx = elem + j;
+    }
+}
 
 // Running sum of exponentials of one thread, relative to a reference logit m that is one of the
 // thread's own elements (or -inf while it has seen none).  fp32 keeps full relative precision
@@ -103,8 +128,12 @@ __device__ __forceinline__ void add_chunk(const uint4 &w, float nmh, Online &st)
 // Adds this thread's chunks (ct, ct + NT, ...) of a stage holding n chunks to its running sum.
 // Four chunks are fetched before any is used; the last, partial group of up to three is fetched
 // together as well.
-template <typename T, int kF>
-__device__ __forceinline__ void add_chunks(uint32_t a0, int n, int ct, int NT, Online &st) {
+// With kArg the running arg max is updated as well (elem0: row-relative element index of the
+// stage's chunk 0).
+template <typename T, int kF, bool kArg>
+__device__ __forceinline__ void add_chunks(uint32_t a0, int n, int ct, int NT, Online &st,
+                                           int elem0, ArgTrack &at) {
+    constexpr int EPC = Elem<T>::kPerChunk;
     const float nmh = -st.mh;
     const uint32_t step = (uint32_t)NT * 16;
     uint32_t a = a0 + (uint32_t)ct * 16;
@@ -112,6 +141,12 @@ __device__ __forceinline__ void add_chunks(uint32_t a0, int n, int ct, int NT, O
     for (; c + 3 * NT < n; c += 4 * NT, a += 4 * step) {
         const uint4 w0 = lds128(a), w1 = lds128(a + step), w2 = lds128(a + 2 * step),
                     w3 = lds128(a + 3 * step);
+        if (kArg) {
+            track_chunk<T>(w0, elem0 + c * EPC, at);
+            track_chunk<T>(w1, elem0 + (c + NT) * EPC, at);
+            track_chunk<T>(w2, elem0 + (c + 2 * NT) * EPC, at);
+            track_chunk<T>(w3, elem0 + (c + 3 * NT) * EPC, at);
+        }
         add_chunk<T, kF>(w0, nmh, st);
         add_chunk<T, kF>(w1, nmh, st);
         add_chunk<T, kF>(w2, nmh, st);
@@ -123,14 +158,20 @@ __device__ __forceinline__ void add_chunks(uint32_t a0, int n, int ct, int NT, O
         uint4 w1 = w0, w2 = w0;
         if (h1) w1 = lds128(a + step);
         if (h2) w2 = lds128(a + 2 * step);
+        if (kArg) {
+            track_chunk<T>(w0, elem0 + c * EPC, at);
+            if (h1) track_chunk<T>(w1, elem0 + (c + NT) * EPC, at);
+            if (h2) track_chunk<T>(w2, elem0 + (c + 2 * NT) * EPC, at);
+        }
         add_chunk<T, kF>(w0, nmh, st);
         if (h1) add_chunk<T, kF>(w1, nmh, st);
         if (h2) add_chunk<T, kF>(w2, nmh, st);
     }
 }
 
-template <typename T, int kF>
-__device__ __forceinline__ void consume_stage(uint32_t a0, int n, int ct, int NT, Online &st) {
+template <typename T, int kF, bool kArg>
+__device__ __forceinline__ void consume_stage(uint32_t a0, int n, int ct, int NT, Online &st,
+                                              int elem0, ArgTrack &at) {
     if (ct >= n) return;
     if (!(st.m > -INFINITY)) {
         // no reference yet (start of a row): the largest element of the first chunk
@@ -138,7 +179,7 @@ __device__ __forceinline__ void consume_stage(uint32_t a0, int n, int ct, int NT
         if (cm > -INFINITY) { st.m = cm; st.mh = cm * kLog2e; }
     }
     const Online saved = st;
-    add_chunks<T, kF>(a0, n, ct, NT, st);
+    add_chunks<T, kF, kArg>(a0, n, ct, NT, st, elem0, at);
     if (!(st.total() < kSumLimit)) {
         // an element far above the reference, a NaN or +inf, or only -inf so far: redo the
         // stage relative to the maximum of this thread's chunks
@@ -146,7 +187,7 @@ __device__ __forceinline__ void consume_stage(uint32_t a0, int n, int ct, int NT
         float cm = -INFINITY;
         for (int c = ct; c < n; c += NT) cm = fmaxf(cm, chunk_max<T>(lds128(a0 + (uint32_t)c * 16)));
         if (cm > st.m) st.raise_to(cm);
-        if (st.m > -INFINITY) add_chunks<T, kF>(a0, n, ct, NT, st);
+        if (st.m > -INFINITY) add_chunks<T, kF, kArg>(a0, n, ct, NT, st, elem0, at);
     }
 }
 
@@ -160,7 +201,7 @@ __device__ __forceinline__ float2 warp_merge(const Online &st) {
     return make_float2(M, Sw);
 }
 
-template <typename T, int kF>
+template <typename T, int kF, bool kArg>
 __global__ void __launch_bounds__(544, 1) verify_rows_tma(const VerifyParams p) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     constexpr int ES = Elem<T>::kBytes, EPC = Elem<T>::kPerChunk;
@@ -263,6 +304,7 @@ __global__ void __launch_bounds__(544, 1) verify_rows_tma(const VerifyParams p) 
                         desc[s].nchunks = pc1 - pc0;
                         desc[s].flags = (part == parts - 1) ? kFlagLast : 0u;
                         desc[s].slot = slot;
+                        desc[s].elem0 = (int32_t)(((int64_t)pc0 * 16 - (int64_t)(g0 - f0)) / ES);
                         const uint32_t bar = full0 + s * 8;
                         if (b1 > b0) {
                             const uint32_t bytes = (uint32_t)(b1 - b0) << 4;
@@ -300,6 +342,8 @@ __global__ void __launch_bounds__(544, 1) verify_rows_tma(const VerifyParams p) 
         const int ct = cw * 32 + lane, NT = CW * 32;
         Online st;
         st.reset();
+        ArgTrack at;
+        at.reset();
         bool failed = false;
         int s = 0;
         uint32_t ph = 0;
@@ -308,14 +352,25 @@ __global__ void __launch_bounds__(544, 1) verify_rows_tma(const VerifyParams p) 
             const int n = desc[s].nchunks;
             const uint32_t flags = desc[s].flags;
             if (flags & kFlagEnd) break;
-            consume_stage<T, kF>(stage0 + (uint32_t)s * p.stage_bytes, n, ct, NT, st);
+            consume_stage<T, kF, kArg>(stage0 + (uint32_t)s * p.stage_bytes, n, ct, NT, st,
+                                       kArg ? desc[s].elem0 : 0, at);
             int64_t slot = 0;
             if (flags & kFlagLast) slot = desc[s].slot;
             __syncwarp();
             if (lane == 0) mbar_arrive(empty0 + s * 8);
             if (flags & kFlagLast) {
                 const float2 r = warp_merge(st);
-                if (lane == 0) p.partials[slot + cw] = r;
+                if (kArg) {
+                    // warp arg max: largest value, lowest index among the lanes that hold it
+                    const float vm = warp_max(at.vmax);
+                    const int vi = __reduce_min_sync(0xffffffffu, at.vmax == vm ? at.vidx : INT_MAX);
+                    if (lane == 0)
+                        reinterpret_cast<float4 *>(p.partials)[slot + cw] =
+                            make_float4(r.x, r.y, vm, __int_as_float(vi));
+                    at.reset();
+                } else {
+                    if (lane == 0) p.partials[slot + cw] = r;
+                }
                 st.reset();
             }
             if (++s == S) { s = 0; ph ^= 1u; }
@@ -440,6 +495,46 @@ __global__ void __launch_bounds__(kFinishThreads) verify_finish_kernel(
     }
 }
 
+// Greedy step: merges the partials of a row, one warp per row.  A partial is
+// (reference, sum, largest logit, index of its first occurrence).
+constexpr int kGreedyWarps = 8;
+__global__ void __launch_bounds__(kGreedyWarps * 32) greedy_finish_kernel(
+    int V, int64_t R, const float4 *__restrict__ partials, int P, int32_t *__restrict__ next_token,
+    float *__restrict__ next_logp, float *__restrict__ row_lse, uint32_t *__restrict__ row_status,
+    const unsigned long long *err_word, unsigned long long epoch) {
+    pdl_enter();
+    const int lane = threadIdx.x & 31;
+    const int64_t r = (int64_t)blockIdx.x * kGreedyWarps + (threadIdx.x >> 5);
+    if (r >= R) return;
+    const float4 *pp = partials + r * P;
+    float Mx = kNegInit, vm = -INFINITY;
+    for (int q = lane; q < P; q += 32) {
+        const float4 v = pp[q];
+        Mx = fmaxf(Mx, v.x);
+        vm = fmaxf(vm, v.z);
+    }
+    Mx = warp_max(Mx);
+    vm = warp_max(vm);
+    float S = 0.f;
+    int vi = INT_MAX;
+    for (int q = lane; q < P; q += 32) {
+        const float4 v = pp[q];
+        S += v.y * ex2((v.x - Mx) * kLog2e);
+        if (v.z == vm) vi = min(vi, __float_as_int(v.w));
+    }
+    S = warp_sum(S);
+    vi = __reduce_min_sync(0xffffffffu, vi);
+    if (lane == 0) {
+        const float lse = Mx + logf(S);
+        uint32_t st = (*err_word == epoch) ? (uint32_t)SSD_UTT_INTERNAL : 0u;
+        if (!(fabsf(lse) < INFINITY)) st |= SSD_UTT_NONFINITE;
+        next_token[r] = (vi < 0 || vi >= V) ? 0 : vi;
+        if (next_logp) next_logp[r] = vm - lse;
+        if (row_lse) row_lse[r] = lse;
+        if (row_status) row_status[r] = st;
+    }
+}
+
 }  // namespace
 
 unsigned long long next_epoch();
@@ -530,11 +625,12 @@ int launch_verify(const void *logits, ssd_dtype dtype, int V, int64_t ld, int64_
             if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
         }
         if (plan.kernel == 2) {
-            void (*kern)(const VerifyParams) = verify_rows_tma<float, 0>;
+            void (*kern)(const VerifyParams) = verify_rows_tma<float, 0, false>;
             if (dtype == SSD_BF16)
-                kern = plan.fma_exp == 1 ? verify_rows_tma<bf16_t, 1>
-                     : plan.fma_exp == 2 ? verify_rows_tma<bf16_t, 2>
-                     : plan.fma_exp == 3 ? verify_rows_tma<bf16_t, 3> : verify_rows_tma<bf16_t, 0>;
+                kern = plan.fma_exp == 1 ? verify_rows_tma<bf16_t, 1, false>
+                     : plan.fma_exp == 2 ? verify_rows_tma<bf16_t, 2, false>
+                     : plan.fma_exp == 3 ? verify_rows_tma<bf16_t, 3, false>
+                                         : verify_rows_tma<bf16_t, 0, false>;
             e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)plan.smem_bytes);
             if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
@@ -563,6 +659,54 @@ int launch_verify(const void *logits, ssd_dtype dtype, int V, int64_t ld, int64_
                    reject_none, skip, static_cast<const float2 *>(partials), plan.partials,
                    token_logp, row_lse, accepted_len, all_accepted, utt_status,
                    static_cast<const unsigned long long *>(err_word), epoch);
+    if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
+    e = cudaGetLastError();
+    if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
+    return SSD_OK;
+}
+
+size_t greedy_workspace_bytes(int64_t R, const VerifyPlan &plan) {
+    return 256 + (size_t)R * plan.partials * sizeof(float4);
+}
+
+int launch_greedy(const void *logits, ssd_dtype dtype, int V, int64_t ld, int64_t R,
+                  void *workspace, int32_t *next_token, float *next_logp, float *row_lse,
+                  uint32_t *row_status, const VerifyPlan &plan, const Launch &L) {
+    if (R == 0) return SSD_OK;
+    if (plan.kernel != 2) return SSD_ERR_ARG;      // only the bulk-copy kernel tracks the arg max
+    const ssd_launch_opts *o = L.opts;
+    unsigned long long *err_word = static_cast<unsigned long long *>(workspace);
+    float4 *partials = reinterpret_cast<float4 *>(static_cast<char *>(workspace) + 256);
+    const unsigned long long epoch = next_epoch();
+    VerifyParams p{};
+    p.logits = static_cast<const char *>(logits);
+    p.V = V; p.ld = ld; p.M = R; p.split = plan.split; p.num_items = R * plan.split;
+    p.tok_off = nullptr; p.B = 0; p.skip = nullptr;
+    p.partials = reinterpret_cast<float2 *>(partials); p.partials_per_row = plan.partials;
+    p.warps = plan.warps; p.stages = plan.stages; p.stage_bytes = plan.stage_bytes;
+    p.err_word = err_word; p.epoch = epoch;
+    const int64_t ctas = p.num_items < plan.ctas ? p.num_items : plan.ctas;
+    cudaError_t e;
+    if (o && o->ev_begin) {
+        e = cudaEventRecord(static_cast<cudaEvent_t>(o->ev_begin), L.stream);
+        if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
+    }
+    void (*kern)(const VerifyParams) = verify_rows_tma<float, 0, true>;
+    if (dtype == SSD_BF16)
+        kern = plan.fma_exp >= 1 ? verify_rows_tma<bf16_t, 1, true> : verify_rows_tma<bf16_t, 0, true>;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
+    if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
+    e = launch_pdl(kern, (unsigned)ctas, (unsigned)((plan.warps + 1) * 32), plan.smem_bytes,
+                   L.stream, p);
+    if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
+    if (o && o->ev_end) {
+        e = cudaEventRecord(static_cast<cudaEvent_t>(o->ev_end), L.stream);
+        if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
+    }
+    e = launch_pdl(greedy_finish_kernel, (unsigned)((R + kGreedyWarps - 1) / kGreedyWarps),
+                   (unsigned)(kGreedyWarps * 32), 0, L.stream, V, R,
+                   static_cast<const float4 *>(partials), plan.partials, next_token, next_logp,
+                   row_lse, row_status, static_cast<const unsigned long long *>(err_word), epoch);
     if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
     e = cudaGetLastError();
     if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }

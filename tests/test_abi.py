@@ -122,3 +122,37 @@ def test_binding_refuses_host_tensors(lib):
     off = torch.tensor([0, 4], dtype=torch.int64)
     with pytest.raises(ValueError):
         ssd.ssd_ctc_draft(x, off, 0, 4)
+
+
+def test_sweep_assemble_greedy_reject_bad_arguments_on_the_host(lib):
+    p = C.c_void_p
+    f = (C.c_float * 2)(0.5, 0.1)
+    fp = C.cast(f, C.c_void_p)
+    sw = lib.ssd_threshold_sweep
+    assert sw(p(8), p(8), p(8), -1, 4, fp, fp, 2, p(8), p(8), p(8), None, None) == ssd.ERR_ARG
+    assert sw(p(8), p(8), p(8), 2, 4, fp, fp, -1, p(8), p(8), p(8), None, None) == ssd.ERR_ARG
+    assert sw(p(8), p(8), None, 2, 4, fp, fp, 2, p(8), p(8), p(8), None, None) == ssd.ERR_NULL
+    assert sw(p(8), p(8), p(8), 2, 4, None, fp, 2, p(8), p(8), p(8), None, None) == ssd.ERR_NULL
+    assert sw(None, p(8), p(8), 2, 4, fp, fp, 2, p(8), p(8), p(8), None, None) == ssd.ERR_NULL
+    assert sw(p(8), None, p(8), 2, 4, fp, fp, 2, p(8), p(8), p(8), None, None) == ssd.ERR_NULL
+    assert sw(p(8), p(8), p(8), 2, 4, fp, fp, 2, p(8), None, p(8), None, None) == ssd.ERR_NULL
+    asm = lib.ssd_assemble
+    a = [p(8)] * 2 + [3, 9] + [p(8)] * 9 + [None]
+    bad = list(a); bad[2] = -1
+    assert asm(*bad) == ssd.ERR_ARG
+    for i in (1, 4, 5, 6, 8, 9, 10, 11, 12):
+        bad = list(a); bad[i] = None
+        assert asm(*bad) == ssd.ERR_NULL, i
+    gs = lib.ssd_greedy_step
+    ok = [p(8), ssd.BF16, 100, 100, 5, p(8), p(8), p(8), p(8), p(256), 1 << 20, None, None]
+    for i, v, code in ((1, 9, ssd.ERR_DTYPE), (2, 0, ssd.ERR_ARG), (3, 99, ssd.ERR_ARG),
+                       (4, -1, ssd.ERR_ARG), (0, None, ssd.ERR_NULL), (5, None, ssd.ERR_NULL),
+                       (0, p(7), ssd.ERR_ALIGN), (9, None, ssd.ERR_WORKSPACE),
+                       (10, 16, ssd.ERR_WORKSPACE), (9, p(264), ssd.ERR_WORKSPACE)):
+        bad = list(ok); bad[i] = v
+        assert gs(*bad) == code, (i, v)
+    o = ssd.LaunchOpts()
+    o.kernel = 1
+    bad = list(ok); bad[12] = C.byref(o)
+    assert gs(*bad) == ssd.ERR_ARG
+    assert ssd.ssd_greedy_step_workspace_bytes(16, 152064, ssd.BF16) >= 256 + 16 * 16 * 12
