@@ -75,6 +75,38 @@ CONFIGS = {
 }
 
 
+# The paper's own shape (Section 3.1 / 3.2): a 348-symbol character CTC head, 50 frames per
+# second of 5-30 s utterances, batches of length-sorted utterances under a 50,000-token budget,
+# and the two operating points of Table 1.  The value mix follows the table's Open ASR averages:
+# high accuracy (tau_CTC 0.7, tau_SLM 0.2) accepts about 14 % of the utterances at the gate and
+# 47 % at verification; high RTFx (tau_CTC 3.0, tau_SLM 0.1) gates close to all of them.
+CONFIGS[5] = Workload("paper_high_accuracy", B=512, t_dist="lognormal", t_lo=250, t_hi=1500,
+                      V_ctc=348, V_llm=49152, dtype="bf16", max_draft_len=1500, tau_ctc=0.7,
+                      tau_slm=0.2, flat_frac=0.05, confident_frac=0.14,
+                      reject_mode="uniform_or_none", p_no_reject=0.547, seed=5)
+CONFIGS[6] = Workload("paper_high_rtfx", B=512, t_dist="lognormal", t_lo=250, t_hi=1500,
+                      V_ctc=348, V_llm=49152, dtype="bf16", max_draft_len=1500, tau_ctc=3.0,
+                      tau_slm=0.1, boost_lo=3.0, flat_frac=0.0, confident_frac=0.0,
+                      reject_mode="uniform_or_none", p_no_reject=0.3, seed=6)
+MAX_BATCH_TOKENS = 50000
+
+
+def length_sorted_batches(lengths: List[int], max_tokens: int = MAX_BATCH_TOKENS) -> List[List[int]]:
+    """Section 3.2's batching: utterances sorted by length (longest first), packed in order
+    into batches whose total frame count stays within the budget (a batch always takes at least
+    one utterance).  Returns the lengths of each batch."""
+    out, cur, tot = [], [], 0
+    for t in sorted((int(v) for v in lengths), reverse=True):
+        if cur and tot + t > max_tokens:
+            out.append(cur)
+            cur, tot = [], 0
+        cur.append(t)
+        tot += t
+    if cur:
+        out.append(cur)
+    return out
+
+
 def sweep_point(B: int, V_llm: int, dtype: str) -> Workload:
     """One point of the throughput sweep (configuration 4): T = 1000, V_ctc = 1025, 250 draft
     tokens per utterance, generators as configuration 1."""

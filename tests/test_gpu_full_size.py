@@ -124,3 +124,33 @@ def test_configurations_2_and_3_sampled(cuda_device, cfg, n_sample):
     check_sample(w, cb, vb, s1, gate, s2, sample)
     del cb, vb, s1, gate, s2
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("cfg", [5, 6])
+def test_paper_shape_batches(cuda_device, cfg):
+    """The paper's own shape: 348 CTC symbols, length-sorted batches of at most 50,000 frames,
+    at the high-accuracy (5) and the high-RTFx (6) operating point.  First and last batch."""
+    w = synth.CONFIGS[cfg]
+    batches = synth.length_sorted_batches(synth.draw_lengths(w))
+    assert all(sum(b) <= synth.MAX_BATCH_TOKENS for b in batches) and sum(len(b) for b in batches) == w.B
+    assert all(a >= b for bt in batches for a, b in zip(bt, bt[1:]))
+    for lengths in (batches[0], batches[-1]):
+        wb = synth.scaled(w, B=len(lengths))
+        dev = cuda_device
+        cb = synth.make_ctc_batch(wb, dev, lengths)
+        off = cb.frame_off.to(dev)
+        s1 = ssd.ssd_ctc_draft(cb.logits, off, wb.blank_id, wb.max_draft_len)
+        gate = ssd.ssd_entropy_gate(s1["frame_entropy"], off, wb.tau_ctc)
+        torch.cuda.synchronize()
+        K = s1["draft_len"].cpu().tolist()
+        vb = synth.make_verify_batch(wb, K, dev)
+        s2 = ssd.ssd_verify(vb.logits, vb.tok_off.to(dev), vb.draft_ids.to(dev), wb.tau_slm,
+                            skip=gate["gate_accept"])
+        torch.cuda.synchronize()
+        ga = gate["gate_accept"].cpu().numpy().astype(bool)
+        if cfg == 6:
+            assert ga.all()                       # "close to 100 % CTC gating"
+        else:
+            np.testing.assert_array_equal(ga, cb.confident.numpy())
+        sample = pick(np.array(lengths), ga, min(5, len(lengths)))
+        check_sample(wb, cb, vb, s1, gate, s2, sample)
