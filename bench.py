@@ -33,7 +33,7 @@ KERNEL_EVENT_EVERY = 5          # N_SETS and this are coprime: every input set g
 N_SETS = 3                      # distinct input batches rotated through, so no step finds its
                                 # inputs in the 126 MB L2
 TRAFFIC_FILE = os.path.join(ROOT, "paper_2603_11243_b200", "ncu_traffic.json")
-KERNEL_SOURCES = ["ssd_common.cuh", "ssd_ctc.cu", "ssd_verify.cu", "ssd_api.cu"]
+KERNEL_SOURCES = ["ssd_common.cuh", "ssd_stream.cuh", "ssd_ctc.cu", "ssd_verify.cu", "ssd_api.cu"]
 
 
 def parse_args():
@@ -401,7 +401,35 @@ def time_next_rows(sets, device, peak):
     t_gk = statistics.mean(kev[2 * j].elapsed_time(kev[2 * j + 1]) for j in range(2, 12)) * 1e3
     w = sets[0]["w"]
     gbytes = R * w.V_llm * (2 if w.dtype == "bf16" else 4)
-    return {"threshold_sweep": {"pairs": len(pairs), "us_per_call": round(t_sw, 2)},
+    # the whole step with ssd_verify_early_exit in place of ssd_verify (same decisions; the
+    # per-token log-likelihoods only up to a little past each first reject)
+    code = ssd.BF16 if w.dtype == "bf16" else ssd.F32
+    ee = []
+    for s in sets:
+        o = ssd.alloc_early_exit_outputs(s["M"], s["B"], s["w"].V_llm, code, device)
+        ee.append((ssd.bind_verify_early_exit(s["vb"].logits, s["tok_off"], s["ids"],
+                                              s["w"].tau_slm, o, skip=s["gate"]["gate_accept"]), o))
+
+    def ee_step(i):
+        sets[i]["call_ctc"]()
+        sets[i]["call_gate"]()
+        ee[i][0]()
+
+    n_ee = max(20, min(400, int(0.05 / max(1e-6, sum(s["verify_bytes"] for s in sets) / n_sets / 5e12))))
+    t_ee = timed(ee_step, n_ee)
+    same = all(torch.equal(ee[i][1]["accepted_len"], sets[i]["s2"]["accepted_len"]) and
+               torch.equal(ee[i][1]["all_accepted"], sets[i]["s2"]["all_accepted"])
+               for i in range(n_sets))
+    rows_read = sum(int(ee[i][1]["rows_read"].clamp(min=0).sum().item()) for i in range(n_sets))
+    fell_back = any(bool((ee[i][1]["rows_read"] < 0).any().item()) for i in range(n_sets))
+    rows_full = sum(s["m_active"] for s in sets)
+    units = sum(s["B"] for s in sets) / n_sets
+    early = {"utterances_per_s": round(units / (t_ee * 1e-6), 1), "us_per_step": round(t_ee, 2),
+             "verify_rows_read_frac": None if fell_back else round(rows_read / max(rows_full, 1), 4),
+             "same_decisions_as_full": bool(same),
+             "note": "separate mode, not part of `value`: rows after an utterance's first reject "
+                     "are not read (Section 2.3 needs only the first reject)"}
+    return {"early_exit_step": early, "threshold_sweep": {"pairs": len(pairs), "us_per_call": round(t_sw, 2)},
             "assemble": {"us_per_call": round(t_asm, 2),
                          "ar_count": int(prep[0][1]["ar_count"].cpu()[0])},
             "greedy_step": {"rows": R, "V": w.V_llm, "us_per_call": round(t_gr, 2),

@@ -179,6 +179,33 @@ int32_t ssd_verify(const void *logits, ssd_dtype dtype, int32_t V, int64_t ld,
                    const ssd_launch_opts *opts);
 
 /*
+ * ssd_verify that stops reading an utterance once its first rejected position is known.
+ * Section 2.3 of the paper needs only j, the FIRST position whose likelihood is <= tau_SLM:
+ * the rows after it cannot change the decision.  Rows are visited position by position across
+ * all utterances; a row is skipped when a smaller rejected position of its utterance has
+ * already been found.  accepted_len, all_accepted and utt_status are exactly those of
+ * ssd_verify (status bits only reflect the rows that were read).  token_logp / row_lse are
+ * written for every row that was read -- always including positions 0 .. accepted_len[b] --
+ * and left untouched for the others; which later rows still get read depends on timing.
+ *   rows_read[b] (nullable, [B] i32): rows of utterance b that were read; -1 for every
+ *   utterance when the call fell back to the full kernel (fewer than four rows per CTA, or
+ *   column spans in use), which reads all rows of every verified utterance.
+ * Use ssd_verify when the complete token_logp is wanted (e.g. for ssd_threshold_sweep).
+ * workspace: at least ssd_verify_early_exit_workspace_bytes(...) bytes, 256-byte aligned.
+ * Errors: as ssd_verify.
+ */
+size_t ssd_verify_early_exit_workspace_bytes(int32_t B, int64_t M, int32_t V, ssd_dtype dtype,
+                                             const ssd_launch_opts *opts);
+int32_t ssd_verify_early_exit(const void *logits, ssd_dtype dtype, int32_t V, int64_t ld,
+                              const int64_t *tok_off, const int32_t *draft_ids, int32_t B,
+                              int64_t M, float tau_slm, const uint8_t *skip,
+                              float *token_logp, float *row_lse,
+                              int32_t *accepted_len, uint8_t *all_accepted, uint32_t *utt_status,
+                              int32_t *rows_read,
+                              void *workspace, size_t workspace_bytes, void *stream,
+                              const ssd_launch_opts *opts);
+
+/*
  * Operating points from one pass.  Section 3.2 of the paper studies tau_CTC in [0.7, 3.0] and
  * tau_SLM in {0.1, 0.2} (Table 1 gives two of the points); both decisions depend on the logits
  * only through the per-utterance maximum entropy (Eq. 3) and the per-token log-likelihoods

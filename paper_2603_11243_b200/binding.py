@@ -67,6 +67,11 @@ def lib():
         L.ssd_verify_static.restype = i32
         L.ssd_verify_static.argtypes = [vp, C.c_int, i32, i64, vp, vp, i32, i64, C.c_float, vp,
                                         vp, vp, vp, vp, vp, vp, vp]
+        L.ssd_verify_early_exit_workspace_bytes.restype = C.c_size_t
+        L.ssd_verify_early_exit_workspace_bytes.argtypes = [C.c_int32, C.c_int64, C.c_int32, C.c_int, C.c_void_p]
+        L.ssd_verify_early_exit.restype = i32
+        L.ssd_verify_early_exit.argtypes = [vp, C.c_int, i32, i64, vp, vp, i32, i64, C.c_float, vp,
+                                            vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp, vp]
         L.ssd_threshold_sweep.restype = i32
         L.ssd_threshold_sweep.argtypes = [vp, vp, vp, i32, i64, vp, vp, i32, vp, vp, vp, vp, vp]
         L.ssd_assemble.restype = i32
@@ -240,6 +245,59 @@ def ssd_verify_static(logits: torch.Tensor, tok_off: torch.Tensor, draft_ids: to
     if rc != OK:
         raise SsdError(rc, "ssd_verify_static")
     return out
+
+
+def ssd_verify_early_exit_workspace_bytes(B, M, V, dtype_code, opts=None) -> int:
+    return int(lib().ssd_verify_early_exit_workspace_bytes(B, M, V, dtype_code, _opts(opts)))
+
+
+def _early_exit_args(logits, tok_off, draft_ids, tau_slm, out, skip, V, opts):
+    M, ld = _rows_ld(logits)
+    V = logits.shape[1] if V is None else V
+    B = tok_off.shape[0] - 1
+    if tok_off.dtype != torch.int64 or draft_ids.dtype != torch.int32:
+        raise TypeError("tok_off must be int64 and draft_ids int32")
+    if skip is not None and skip.dtype != torch.uint8:
+        raise TypeError("skip must be uint8")
+    ws = out["workspace"]
+    return [_dev(logits, "logits"), _dtype_code(logits), V, ld, _dev(tok_off, "tok_off"),
+            _dev(draft_ids, "draft_ids"), B, M, C.c_float(tau_slm), _dev(skip, "skip"),
+            _dev(out["token_logp"], "token_logp"), _dev(out.get("row_lse"), "row_lse"),
+            _dev(out["accepted_len"], "accepted_len"), _dev(out["all_accepted"], "all_accepted"),
+            _dev(out["utt_status"], "utt_status"), _dev(out.get("rows_read"), "rows_read"),
+            _dev(ws, "workspace"), ws.numel(), _stream(), _opts(opts)]
+
+
+def alloc_early_exit_outputs(M, B, V, dtype_code, device, opts=None) -> Dict[str, torch.Tensor]:
+    out = alloc_verify_outputs(M, B, device,
+                               ssd_verify_early_exit_workspace_bytes(B, M, V, dtype_code, opts))
+    out["rows_read"] = torch.empty((B,), dtype=torch.int32, device=device)
+    return out
+
+
+def ssd_verify_early_exit(logits: torch.Tensor, tok_off: torch.Tensor, draft_ids: torch.Tensor,
+                          tau_slm: float, skip: Optional[torch.Tensor] = None,
+                          V: Optional[int] = None, out=None,
+                          opts: Optional[LaunchOpts] = None) -> Dict[str, torch.Tensor]:
+    """Stage 2 with early exit (Section 2.3 needs only the first reject): same decisions as
+    ssd_verify; token_logp only for the rows that were read."""
+    if out is None:
+        M = logits.shape[0]
+        out = alloc_early_exit_outputs(M, tok_off.shape[0] - 1,
+                                       logits.shape[1] if V is None else V, _dtype_code(logits),
+                                       logits.device, opts)
+    rc = lib().ssd_verify_early_exit(*_early_exit_args(logits, tok_off, draft_ids, tau_slm, out,
+                                                       skip, V, opts))
+    if rc != OK:
+        raise SsdError(rc, "ssd_verify_early_exit")
+    return out
+
+
+def bind_verify_early_exit(logits, tok_off, draft_ids, tau_slm, out, skip=None, V=None,
+                           opts: Optional[LaunchOpts] = None):
+    args = _early_exit_args(logits, tok_off, draft_ids, tau_slm, out, skip, V, opts)
+    return BoundCall(lib().ssd_verify_early_exit, "ssd_verify_early_exit", args,
+                     (logits, tok_off, draft_ids, out, skip, opts), True)
 
 
 def ssd_threshold_sweep(utt_max_entropy: torch.Tensor, token_logp: torch.Tensor,

@@ -142,6 +142,52 @@ int32_t ssd_assemble(const int32_t *tokens, const int64_t *tok_off, int32_t B, i
                            static_cast<cudaStream_t>(stream));
 }
 
+size_t ssd_verify_early_exit_workspace_bytes(int32_t B, int64_t M, int32_t V, ssd_dtype dtype,
+                                             const ssd_launch_opts *opts) {
+    if (B < 0 || M < 0 || V < 1 || (dtype != SSD_F32 && dtype != SSD_BF16)) return 0;
+    VerifyPlan plan;
+    if (plan_verify(B, M, V, dtype, opts, &plan) != SSD_OK) return 0;
+    return verify_ee_workspace_bytes(B, plan);
+}
+
+int32_t ssd_verify_early_exit(const void *logits, ssd_dtype dtype, int32_t V, int64_t ld,
+                              const int64_t *tok_off, const int32_t *draft_ids, int32_t B,
+                              int64_t M, float tau_slm, const uint8_t *skip,
+                              float *token_logp, float *row_lse,
+                              int32_t *accepted_len, uint8_t *all_accepted, uint32_t *utt_status,
+                              int32_t *rows_read,
+                              void *workspace, size_t workspace_bytes, void *stream,
+                              const ssd_launch_opts *opts) {
+    if (dtype != SSD_F32 && dtype != SSD_BF16) return SSD_ERR_DTYPE;
+    if (B < 0 || M < 0 || V < 1 || ld < V) return SSD_ERR_ARG;
+    if (!tok_off) return SSD_ERR_NULL;
+    if (M > 0 && (!logits || !draft_ids || !token_logp)) return SSD_ERR_NULL;
+    if (B > 0 && (!accepted_len || !all_accepted || !utt_status)) return SSD_ERR_NULL;
+    const int es = dtype == SSD_F32 ? 4 : 2;
+    if (reinterpret_cast<uintptr_t>(logits) % es) return SSD_ERR_ALIGN;
+    VerifyPlan plan;
+    int rc = plan_verify(B, M, V, dtype, opts, &plan);
+    if (rc != SSD_OK) return rc;
+    if (B > 0 && (!workspace || workspace_bytes < verify_ee_workspace_bytes(B, plan) ||
+                  reinterpret_cast<uintptr_t>(workspace) % 256))
+        return SSD_ERR_WORKSPACE;
+    Launch L{static_cast<cudaStream_t>(stream), opts};
+    if (!verify_ee_applicable(B, M, plan)) {
+        // too few rows to deal out position by position: the full kernel, whose outputs
+        // are a superset; every row of a verified utterance is then read
+        rc = launch_verify(logits, dtype, V, ld, M, tok_off, draft_ids, B, tau_slm, skip, workspace,
+                           token_logp, row_lse, accepted_len, all_accepted, utt_status, plan, L);
+        if (rc == SSD_OK && rows_read && B > 0) {
+            cudaError_t e = cudaMemsetAsync(rows_read, 0xff, (size_t)B * sizeof(int32_t), L.stream);
+            if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
+        }
+        return rc;
+    }
+    return launch_verify_ee(logits, dtype, V, ld, M, tok_off, draft_ids, B, tau_slm, skip, workspace,
+                            token_logp, row_lse, accepted_len, all_accepted, utt_status, rows_read,
+                            plan, L);
+}
+
 size_t ssd_greedy_step_workspace_bytes(int64_t R, int32_t V, ssd_dtype dtype,
                                        const ssd_launch_opts *opts) {
     if (R < 0 || V < 1 || (dtype != SSD_F32 && dtype != SSD_BF16)) return 0;

@@ -355,6 +355,14 @@ int launch_assemble(const int32_t *tokens, const int64_t *tok_off, int B, int64_
                     uint8_t *is_final, int32_t *ar_count, int32_t *ar_utt, int32_t *ar_resume,
                     cudaStream_t stream);
 
+size_t verify_ee_workspace_bytes(int B, const VerifyPlan &full_plan);
+bool verify_ee_applicable(int B, int64_t M, const VerifyPlan &plan);
+int launch_verify_ee(const void *logits, ssd_dtype dtype, int V, int64_t ld, int64_t M,
+                     const int64_t *tok_off, const int32_t *draft_ids, int B, float tau_slm,
+                     const uint8_t *skip, void *workspace, float *token_logp, float *row_lse,
+                     int32_t *accepted_len, uint8_t *all_accepted, uint32_t *utt_status,
+                     int32_t *rows_read, const VerifyPlan &plan, const Launch &L);
+
 void record_cuda_error(cudaError_t e);
 
 }  // namespace ssd

@@ -156,3 +156,20 @@ def test_sweep_assemble_greedy_reject_bad_arguments_on_the_host(lib):
     bad = list(ok); bad[12] = C.byref(o)
     assert gs(*bad) == ssd.ERR_ARG
     assert ssd.ssd_greedy_step_workspace_bytes(16, 152064, ssd.BF16) >= 256 + 16 * 16 * 12
+
+
+def test_early_exit_rejects_bad_arguments_on_the_host(lib):
+    p = C.c_void_p
+    ee = lib.ssd_verify_early_exit
+    ok = [p(8), ssd.BF16, 100, 100, p(8), p(8), 2, 40, C.c_float(0.1), None, p(8), p(8), p(8), p(8),
+          p(8), None, p(256), 1 << 20, None, None]
+    for i, v, code in ((1, 4, ssd.ERR_DTYPE), (2, 0, ssd.ERR_ARG), (3, 50, ssd.ERR_ARG),
+                       (6, -1, ssd.ERR_ARG), (7, -1, ssd.ERR_ARG), (0, None, ssd.ERR_NULL),
+                       (4, None, ssd.ERR_NULL), (5, None, ssd.ERR_NULL), (10, None, ssd.ERR_NULL),
+                       (12, None, ssd.ERR_NULL), (0, p(7), ssd.ERR_ALIGN),
+                       (16, None, ssd.ERR_WORKSPACE), (17, 64, ssd.ERR_WORKSPACE),
+                       (16, p(257), ssd.ERR_WORKSPACE)):
+        bad = list(ok); bad[i] = v
+        assert ee(*bad) == code, (i, v)
+    full = ssd.ssd_verify_workspace_bytes(64, 20000, 49152, ssd.BF16)
+    assert ssd.ssd_verify_early_exit_workspace_bytes(64, 20000, 49152, ssd.BF16) >= full

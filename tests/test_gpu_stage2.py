@@ -183,3 +183,100 @@ def test_runs_are_bit_identical(cuda_device):
     b = run_verify(x, vb.tok_off, vb.draft_ids, w.V_llm, 0.1, guard=False)
     for k in ("token_logp", "row_lse", "accepted_len", "all_accepted"):
         assert torch.equal(a[k], b[k]), k
+
+
+# ---- early exit --------------------------------------------------------------------------------
+
+def check_early_exit(w, K, device, skip=None, **okw):
+    """ssd_verify_early_exit against the oracle and against ssd_verify: identical decisions,
+    log-likelihoods for every position up to the first reject, untouched or correct beyond."""
+    vb = synth.make_verify_batch(w, K, "cpu")
+    x, off, ids = vb.logits.to(device), vb.tok_off.to(device), vb.draft_ids.to(device)
+    o = H.opts(**okw) if okw else None
+    code = ssd.BF16 if x.dtype == torch.bfloat16 else ssd.F32
+    out = ssd.alloc_early_exit_outputs(x.shape[0], len(K), w.V_llm, code, device, o)
+    out["token_logp"].fill_(float("nan"))
+    out["row_lse"].fill_(float("nan"))
+    skip_dev = None if skip is None else torch.as_tensor(skip, dtype=torch.uint8).to(device)
+    ssd.ssd_verify_early_exit(x, off, ids, w.tau_slm, skip=skip_dev, out=out, opts=o)
+    torch.cuda.synchronize()
+    orc = ref.verify(H.storage_numpy(vb.logits), w.V_llm, vb.tok_off.numpy(), vb.draft_ids.numpy(),
+                     float(np.float32(w.tau_slm)), skip=skip)
+    np.testing.assert_array_equal(out["accepted_len"].cpu().numpy(), orc["accepted_len"])
+    np.testing.assert_array_equal(out["all_accepted"].cpu().numpy(), orc["all_accepted"])
+    lp, lse = out["token_logp"].cpu().numpy(), out["row_lse"].cpu().numpy()
+    rr = out["rows_read"].cpu().numpy()
+    toff = vb.tok_off.numpy()
+    for b in range(len(K)):
+        if skip is not None and skip[b]:
+            assert rr[b] in (0, -1) and np.isnan(lp[toff[b]:toff[b + 1]]).all()
+            continue
+        need = min(K[b], int(orc["accepted_len"][b]) + 1)
+        seg, want = lp[toff[b]:toff[b + 1]].astype(np.float64), orc["token_logp"][toff[b]:toff[b + 1]]
+        assert not np.isnan(seg[:need]).any(), "a position up to the first reject was not read"
+        read = ~np.isnan(seg)
+        assert np.abs(seg[read] - want[read]).max(initial=0.0) <= H.FLOAT_TOL
+        ls = lse[toff[b]:toff[b + 1]].astype(np.float64)
+        assert np.abs(ls[read] - orc["row_lse"][toff[b]:toff[b + 1]][read]).max(initial=0.0) <= H.FLOAT_TOL
+        if rr[b] >= 0:
+            assert rr[b] == read.sum() and need <= rr[b] <= K[b]
+    return vb, out, orc, rr
+
+
+def test_early_exit_reads_fewer_rows_and_decides_the_same(cuda_device):
+    """Enough rows for the position-major kernel (>= 4 per CTA): planted rejects at all depths."""
+    w = synth.scaled(synth.CONFIGS[3], B=24, V_llm=8192, seed=71)          # reject at f*K, f~U(0,1)
+    K = [300 + 7 * (i % 11) for i in range(24)]        # ~50 rows per CTA: the lag of a few rows
+                                                       # per CTA leaves most of the saving
+    vb, out, orc, rr = check_early_exit(w, K, cuda_device)
+    assert (rr >= 0).all()
+    want = [int(p) if p >= 0 else k for p, k in zip(vb.planted_reject.tolist(), K)]
+    assert list(orc["accepted_len"]) == want
+    assert rr.sum() < 0.85 * sum(K), "rows after the first reject were not skipped"
+    full = ssd.ssd_verify(vb.logits.to(cuda_device), vb.tok_off.to(cuda_device),
+                          vb.draft_ids.to(cuda_device), w.tau_slm)
+    torch.cuda.synchronize()
+    assert torch.equal(full["accepted_len"], out["accepted_len"])
+    assert torch.equal(full["utt_status"], out["utt_status"])
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("V", [17, 5003, 49152])
+def test_early_exit_shapes_skip_and_ragged(cuda_device, dtype, V):
+    w = synth.scaled(synth.CONFIGS[1], B=9, V_llm=V, dtype=dtype, seed=300 + V % 89)
+    K = [70, 0, 91, 1, 66, 80, 75, 99, 120]
+    skip = np.array([0, 0, 1, 0, 0, 0, 1, 0, 0], np.uint8)
+    check_early_exit(w, K, cuda_device, skip=skip)
+    check_early_exit(w, K, cuda_device, skip=None, warps=4, stages=3, stage_bytes=4096, ctas=7)
+
+
+def test_early_exit_falls_back_on_small_batches(cuda_device):
+    w = synth.scaled(synth.CONFIGS[1], B=3, V_llm=32000, seed=9)
+    vb, out, orc, rr = check_early_exit(w, [12, 30, 7], cuda_device)
+    assert (rr == -1).all()
+    assert not np.isnan(out["token_logp"].cpu().numpy()).any()        # the full kernel read everything
+
+
+def test_early_exit_bad_ids_nonfinite_and_thresholds(cuda_device):
+    V, B, Kb = 300, 8, 90
+    g = torch.Generator().manual_seed(12)
+    x = torch.randn((B * Kb, V), generator=g)
+    ids = torch.randint(0, V, (B * Kb,), generator=g, dtype=torch.int32)
+    x[torch.arange(B * Kb), ids.long()] += 14.0
+    off = torch.arange(0, B * Kb + 1, Kb, dtype=torch.int64)
+    bad = ids.clone()
+    bad[1 * Kb + 5] = V            # utterance 1: out-of-range id at position 5
+    x2 = x.clone()
+    x2[2 * Kb + 0, 3] = float("nan")   # utterance 2: NaN in its first row
+    dev = cuda_device
+    out = ssd.ssd_verify_early_exit(x2.to(dev), off.to(dev), bad.to(dev), 0.1)
+    torch.cuda.synchronize()
+    st = H.status_u32(out["utt_status"])
+    assert st[1] & ssd.UTT_BAD_DRAFT_ID and st[2] & ssd.UTT_NONFINITE
+    acc = out["accepted_len"].cpu().tolist()
+    assert acc[1] == 5 and acc[2] == 0 and acc[0] == Kb and acc[3:] == [Kb] * 5
+    none = ssd.ssd_verify_early_exit(x.to(dev), off.to(dev), ids.to(dev), 0.0)
+    every = ssd.ssd_verify_early_exit(x.to(dev), off.to(dev), ids.to(dev), 1.0)
+    torch.cuda.synchronize()
+    assert none["accepted_len"].cpu().tolist() == [Kb] * B
+    assert every["accepted_len"].cpu().tolist() == [0] * B
