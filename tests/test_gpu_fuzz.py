@@ -1,0 +1,155 @@
+"""Randomised parity: shapes, paddings, base misalignments, dtypes, ragged lengths, value scales
+and masked (-inf) entries drawn from a seeded generator; every call against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+import helpers as H
+from oracle import ref
+from paper_2603_11243_b200 import binding as ssd
+
+pytestmark = pytest.mark.gpu
+
+
+def random_matrix(rng, rows, V, dtype):
+    """A [rows, V] view into a wider, offset matrix: ld > V and an element-aligned base."""
+    pad, col0 = int(rng.integers(0, 9)), int(rng.integers(0, 8))
+    ld = V + pad + col0
+    scale = float(rng.choice([0.3, 1.0, 4.0, 12.0]))
+    x = rng.normal(size=(rows, ld)).astype(np.float32) * scale
+    if rows and V > 2 and rng.random() < 0.5:            # some masked logits
+        mask = rng.random(size=(rows, ld)) < 0.1
+        mask[:, col0 + int(rng.integers(0, V))] = False  # never a whole row
+        x[mask] = -np.inf
+    t = torch.from_numpy(x).to(dtype)
+    return t, col0, ld
+
+
+def ragged(rng, B, hi):
+    lens = rng.integers(0, hi + 1, size=B)
+    if B > 1:
+        lens[int(rng.integers(0, B))] = 0
+    return np.concatenate([[0], np.cumsum(lens)]).astype(np.int64), lens
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_stage1_random(cuda_device, seed):
+    rng = np.random.default_rng(1000 + seed)
+    V = int(rng.choice([1, 2, 5, 17, 64, 129, 348, 777, 1025, 2051, 4097]))
+    dtype = torch.bfloat16 if rng.random() < 0.5 else torch.float32
+    off, lens = ragged(rng, int(rng.integers(1, 8)), 90)
+    wide, col0, ld = random_matrix(rng, int(off[-1]), V, dtype)
+    blank = int(rng.integers(0, V))
+    cap = int(rng.integers(0, 40))
+    tau = float(rng.uniform(0.05, 4.0))
+    dev = cuda_device
+    view = wide.to(dev)[:, col0:col0 + V]
+    g, out = H.guarded_ctc_outputs(int(off[-1]), len(lens), dev)
+    offd = torch.from_numpy(off).to(dev)
+    ssd.ssd_ctc_draft(view, offd, blank, cap, V=V, out=out)
+    gate = ssd.ssd_entropy_gate(out["frame_entropy"], offd, tau)
+    torch.cuda.synchronize()
+    g.check()
+    orc = H.oracle_stage1(H.storage_numpy(wide[:, col0:col0 + V].contiguous()), V, off, blank, cap, tau)
+    H.compare_stage1(out, gate, orc, off, tau, require_all_margins=False)
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_stage2_random(cuda_device, seed):
+    rng = np.random.default_rng(2000 + seed)
+    V = int(rng.choice([1, 3, 40, 1000, 4099, 20001, 32000, 65537]))
+    dtype = torch.bfloat16 if rng.random() < 0.5 else torch.float32
+    B = int(rng.integers(1, 7))
+    off, lens = ragged(rng, B, 30 if V > 10000 else 120)
+    M = int(off[-1])
+    wide, col0, ld = random_matrix(rng, M, V, dtype)
+    ids = rng.integers(0, V, size=M).astype(np.int32)
+    if M and rng.random() < 0.3:
+        ids[int(rng.integers(0, M))] = V + 3                 # one out-of-range id
+    for r in range(M):                                        # most draft tokens likely
+        if 0 <= ids[r] < V and rng.random() < 0.8:
+            wide[r, col0 + ids[r]] = 25.0
+    tau = float(rng.choice([0.0, 0.05, 0.1, 0.2, 0.9]))
+    skip = (rng.random(size=B) < 0.25).astype(np.uint8) if rng.random() < 0.5 else None
+    dev = cuda_device
+    view = wide.to(dev)[:, col0:col0 + V]
+    code = ssd.BF16 if dtype == torch.bfloat16 else ssd.F32
+    g, out = H.guarded_verify_outputs(M, B, dev, ssd.ssd_verify_workspace_bytes(B, M, V, code))
+    skipd = None if skip is None else torch.from_numpy(skip).to(dev)
+    offd, idsd = torch.from_numpy(off).to(dev), torch.from_numpy(ids).to(dev)
+    ssd.ssd_verify(view, offd, idsd, tau, skip=skipd, V=V, out=out)
+    torch.cuda.synchronize()
+    g.check()
+    orc = ref.verify(H.storage_numpy(wide[:, col0:col0 + V].contiguous()), V, off, ids,
+                     float(np.float32(tau)), skip=skip)
+    H.compare_stage2(out, orc, off, tau, skip=skip, require_all_margins=False)
+    # the early-exit call decides the same (it falls back to the full kernel at these sizes
+    # unless there are many rows)
+    ee = ssd.ssd_verify_early_exit(view, offd, idsd, tau, skip=skipd, V=V)
+    torch.cuda.synchronize()
+    assert torch.equal(ee["accepted_len"], out["accepted_len"])
+    assert torch.equal(ee["all_accepted"], out["all_accepted"])
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_greedy_random(cuda_device, seed):
+    rng = np.random.default_rng(3000 + seed)
+    V = int(rng.choice([1, 2, 33, 1000, 4099, 20001, 49152, 100003]))
+    dtype = torch.bfloat16 if rng.random() < 0.5 else torch.float32
+    R = int(rng.integers(1, 40 if V > 10000 else 300))
+    wide, col0, ld = random_matrix(rng, R, V, dtype)
+    dev = cuda_device
+    out = ssd.ssd_greedy_step(wide.to(dev)[:, col0:col0 + V], V=V)
+    torch.cuda.synchronize()
+    orc = ref.greedy_step(H.storage_numpy(wide[:, col0:col0 + V].contiguous()), V)
+    np.testing.assert_array_equal(out["next_token"].cpu().numpy(), orc["next_token"])
+    assert np.abs(out["next_logp"].cpu().numpy().astype(np.float64) - orc["next_logp"]).max() <= H.FLOAT_TOL
+    assert np.abs(out["row_lse"].cpu().numpy().astype(np.float64) - orc["row_lse"]).max() <= H.FLOAT_TOL
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_early_exit_random_large(cuda_device, seed):
+    """Enough rows for the position-major kernel; random reject structure."""
+    rng = np.random.default_rng(4000 + seed)
+    V = int(rng.choice([257, 4099, 16384]))
+    dtype = torch.bfloat16 if rng.random() < 0.5 else torch.float32
+    B = int(rng.integers(5, 40))
+    lens = rng.integers(20, 140, size=B)
+    lens[int(rng.integers(0, B))] = 0
+    off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    M = int(off[-1])
+    while M < 8 * 148 + 100:                  # below that, rows are cut into column spans
+        lens = lens + 40                      # and the call falls back to the full kernel
+        off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+        M = int(off[-1])
+    wide, col0, ld = random_matrix(rng, M, V, dtype)
+    ids = rng.integers(0, V, size=M).astype(np.int32)
+    for r in range(M):
+        if rng.random() < 0.97:
+            wide[r, col0 + ids[r]] = 25.0
+    tau = 0.1
+    dev = cuda_device
+    view = wide.to(dev)[:, col0:col0 + V]
+    offd, idsd = torch.from_numpy(off).to(dev), torch.from_numpy(ids).to(dev)
+    code = ssd.BF16 if dtype == torch.bfloat16 else ssd.F32
+    out = ssd.alloc_early_exit_outputs(M, B, V, code, dev)
+    out["token_logp"].fill_(float("nan"))
+    ssd.ssd_verify_early_exit(view, offd, idsd, tau, V=V, out=out)
+    torch.cuda.synchronize()
+    orc = ref.verify(H.storage_numpy(wide[:, col0:col0 + V].contiguous()), V, off, ids, float(np.float32(tau)))
+    lp = out["token_logp"].cpu().numpy().astype(np.float64)
+    safe = np.abs(orc["token_logp"] - np.log(tau)) > H.MARGIN
+    for b in range(B):
+        s = slice(int(off[b]), int(off[b + 1]))
+        if not safe[s].all():
+            continue
+        assert int(out["accepted_len"].cpu()[b]) == orc["accepted_len"][b]
+        need = min(int(lens[b]), int(orc["accepted_len"][b]) + 1)
+        seg = lp[s]
+        assert not np.isnan(seg[:need]).any()
+        read = ~np.isnan(seg)
+        want = orc["token_logp"][s]
+        fin = read & np.isfinite(want)
+        assert np.abs(seg[fin] - want[fin]).max(initial=0.0) <= H.FLOAT_TOL
+        np.testing.assert_array_equal(seg[read & ~np.isfinite(want)], want[read & ~np.isfinite(want)])
+    assert (out["rows_read"].cpu().numpy() >= 0).all()
