@@ -193,15 +193,21 @@ __device__ __forceinline__ float fmax_nan_fwd(float a, float b) {
     return d;
 }
 
+__device__ __forceinline__ float fmin_nan(float a, float b) {
+    float d;
+    asm("min.NaN.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+    return d;
+}
+
 // 2^t for a pair, on the FMA pipe: round t to the nearest integer n with the 1.5*2^23 trick,
 // evaluate a degree-4 polynomial for 2^f on f = t - n in [-1/2, 1/2] (relative error 3.6e-6)
-// and add n to the exponent field.  t is clamped to >= -126 first (the result is then at most
-// 2^-126 where the true value is smaller), NaN is kept by the clamp; t >= 128 or NaN give a
-// non-finite or huge value that the callers' range checks catch.
+// and add n to the exponent field.  t is clamped to [-126, 128] first: below, the result is at
+// most 2^-126 where the true value is smaller; above, it is +inf (without the clamp the
+// exponent field would wrap), which the callers' range checks catch.  NaN passes the clamps.
 __device__ __forceinline__ float2 exp2_fma_pair(float2 t) {
     const float kMagic = 12582912.f;
-    t.x = fmax_nan_fwd(t.x, -126.f);
-    t.y = fmax_nan_fwd(t.y, -126.f);
+    t.x = fmin_nan(fmax_nan_fwd(t.x, -126.f), 128.f);
+    t.y = fmin_nan(fmax_nan_fwd(t.y, -126.f), 128.f);
     const float2 r = fadd2(t, make_float2(kMagic, kMagic));
     const float2 n = fadd2(r, make_float2(-kMagic, -kMagic));
     const float2 f = ffma2(n, make_float2(-1.f, -1.f), t);

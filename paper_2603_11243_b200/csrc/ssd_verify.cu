@@ -312,7 +312,8 @@ __global__ void __launch_bounds__(kFinishThreads) verify_finish_kernel(
                 S += v.y * ex2((v.x - Mx) * kLog2e);
             }
         }
-        const float lse = Mx + logf(S);
+        const float lnS = logf(S);
+        const float lse = Mx + lnS;
         if (!(fabsf(lse) < INFINITY)) myflags |= SSD_UTT_NONFINITE;
         const int id = draft_ids[r];
         float logp;
@@ -323,7 +324,7 @@ __global__ void __launch_bounds__(kFinishThreads) verify_finish_kernel(
             reject = true;
         } else {
             const float x = Elem<T>::load(logits + (r * ld + id) * ES);
-            logp = x - lse;
+            logp = (x - Mx) - lnS;      // not x - lse: keeps its accuracy when |x| is large
             reject = reject_none ? false : !(logp > log_tau);   // p <= tau; NaN rejects
         }
         token_logp[r] = logp;
@@ -370,11 +371,12 @@ __global__ void __launch_bounds__(kGreedyWarps * 32) greedy_finish_kernel(
     S = warp_sum(S);
     vi = __reduce_min_sync(0xffffffffu, vi);
     if (lane == 0) {
-        const float lse = Mx + logf(S);
+        const float lnS = logf(S);
+        const float lse = Mx + lnS;
         uint32_t st = (*err_word == epoch) ? (uint32_t)SSD_UTT_INTERNAL : 0u;
         if (!(fabsf(lse) < INFINITY)) st |= SSD_UTT_NONFINITE;
         next_token[r] = (vi < 0 || vi >= V) ? 0 : vi;
-        if (next_logp) next_logp[r] = vm - lse;
+        if (next_logp) next_logp[r] = (vm - Mx) - lnS;
         if (row_lse) row_lse[r] = lse;
         if (row_status) row_status[r] = st;
     }

@@ -146,7 +146,8 @@ __global__ void __launch_bounds__(544, 1) verify_rows_ee(const EeParams p) {
             const float Ssum = warp_sum(v.y * ex2((v.x - Mx) * kLog2e));
             if (lane == 0) {
                 const RowMeta rm = rowmeta[slot];
-                const float lse = Mx + logf(Ssum);
+                const float lnS = logf(Ssum);
+                const float lse = Mx + lnS;
                 uint32_t fl = 0;
                 if (!(fabsf(lse) < INFINITY)) fl |= SSD_UTT_NONFINITE;
                 float logp;
@@ -156,7 +157,7 @@ __global__ void __launch_bounds__(544, 1) verify_rows_ee(const EeParams p) {
                     logp = -INFINITY;
                     reject = true;
                 } else {
-                    logp = sx[slot] - lse;
+                    logp = (sx[slot] - Mx) - lnS;
                     reject = p.reject_none ? false : !(logp > p.log_tau);   // p <= tau; NaN rejects
                 }
                 p.token_logp[rm.row] = logp;

@@ -153,3 +153,49 @@ def test_early_exit_random_large(cuda_device, seed):
         assert np.abs(seg[fin] - want[fin]).max(initial=0.0) <= H.FLOAT_TOL
         np.testing.assert_array_equal(seg[read & ~np.isfinite(want)], want[read & ~np.isfinite(want)])
     assert (out["rows_read"].cpu().numpy() >= 0).all()
+
+
+def _close_scaled(got, want, what):
+    """fp32 outputs of magnitude 1e3..1e5 cannot be within 1e-4 of the fp64 value: allow two
+    fp32 ulps of the value on top of the absolute tolerance."""
+    got, want = np.asarray(got, np.float64), np.asarray(want, np.float64)
+    fin = np.isfinite(want)
+    tol = H.FLOAT_TOL + 2.5e-7 * np.abs(want[fin])
+    assert (np.abs(got[fin] - want[fin]) <= tol).all(), what
+    np.testing.assert_array_equal(got[~fin], want[~fin])
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("scale", [60.0, 400.0, 3.0e4])
+def test_huge_dynamic_range_takes_the_redo_paths(cuda_device, dtype, scale):
+    """Logits hundreds to tens of thousands of nats apart: sums relative to a lane's first
+    element overflow, so the kernels must fall back to their exact two-pass redo."""
+    rng = np.random.default_rng(int(scale))
+    dev = cuda_device
+    V1, V2 = 1025, 20001
+    x1 = torch.from_numpy((rng.normal(size=(70, V1)) * scale).astype(np.float32)).to(dtype)
+    x1[:, :8] = -scale * 4                      # lanes whose first chunk is far below the maximum
+    off = torch.tensor([0, 30, 70], dtype=torch.int64)
+    out = ssd.ssd_ctc_draft(x1.to(dev), off.to(dev), 0, 50)
+    torch.cuda.synchronize()
+    o1 = ref.ctc_draft(H.storage_numpy(x1), V1, off.numpy(), 0, 50)
+    np.testing.assert_array_equal(out["frame_argmax"].cpu().numpy(), o1["frame_argmax"])
+    np.testing.assert_array_equal(out["draft_len"].cpu().numpy(), o1["draft_len"])
+    _close_scaled(out["frame_lse"].cpu().numpy(), o1["frame_lse"], "frame_lse")
+    _close_scaled(out["frame_entropy"].cpu().numpy(), o1["frame_entropy"], "frame_entropy")
+    x2 = torch.from_numpy((rng.normal(size=(40, V2)) * scale).astype(np.float32)).to(dtype)
+    x2[:, :4096] = -scale * 4
+    ids = torch.from_numpy(rng.integers(0, V2, size=40).astype(np.int32))
+    ids[::3] = torch.from_numpy(np.argmax(x2.float().numpy()[::3], axis=1).astype(np.int32))
+    off2 = torch.tensor([0, 15, 40], dtype=torch.int64)
+    v = ssd.ssd_verify(x2.to(dev), off2.to(dev), ids.to(dev), 0.1)
+    gr = ssd.ssd_greedy_step(x2.to(dev))
+    torch.cuda.synchronize()
+    o2 = ref.verify(H.storage_numpy(x2), V2, off2.numpy(), ids.numpy(), float(np.float32(0.1)))
+    _close_scaled(v["row_lse"].cpu().numpy(), o2["row_lse"], "row_lse")
+    _close_scaled(v["token_logp"].cpu().numpy(), o2["token_logp"], "token_logp")
+    np.testing.assert_array_equal(v["accepted_len"].cpu().numpy(), o2["accepted_len"])
+    og = ref.greedy_step(H.storage_numpy(x2), V2)
+    np.testing.assert_array_equal(gr["next_token"].cpu().numpy(), og["next_token"])
+    _close_scaled(gr["next_logp"].cpu().numpy(), og["next_logp"], "next_logp")
+    _close_scaled(gr["row_lse"].cpu().numpy(), og["row_lse"], "greedy row_lse")
