@@ -124,3 +124,56 @@ def test_malformed_offsets_are_flagged_not_followed():
     off = np.array([0, 3, 2, 4], np.int64)  # utterance 1 runs backwards
     o = ref.ctc_draft(x, 3, off, 0, 10)
     assert o["utt_status"][1] == ref.UTT_BAD_OFFSETS and o["draft_len"][1] == 0
+
+
+# ---- the two writings of the definitions against each other, on random inputs ----------------
+
+@pytest.mark.parametrize("seed", range(8))
+def test_c_oracle_and_numpy_oracle_agree_on_random_batches(seed):
+    """Two independently written statements of the same mathematics (sequential C with a
+    two-pass softmax; NumPy through normalised probabilities and run-length groups) must agree
+    on the whole path, bf16 and fp32, ragged batches, every threshold outcome."""
+    from oracle import mini
+    from oracle_impls import to_storage
+    rng = np.random.default_rng(700 + seed)
+    dtype = "bf16" if seed % 2 else "f32"
+    V, B = int(rng.integers(2, 40)), int(rng.integers(1, 6))
+    T = rng.integers(0, 25, size=B)
+    off = np.concatenate([[0], np.cumsum(T)]).astype(np.int64)
+    x = to_storage(rng.normal(size=(int(off[-1]), V)) * rng.choice([0.5, 3.0, 9.0]), dtype)
+    blank, cap, tau_c = int(rng.integers(0, V)), int(rng.integers(1, 12)), float(rng.uniform(0.2, 3.0))
+    o = ref.ctc_draft(x, V, off, blank, cap)
+    g = ref.entropy_gate(o["frame_entropy"], off, tau_c)
+    xw = mini.widen(x).reshape(-1, V)
+    for b in range(B):
+        rows = xw[off[b]:off[b + 1]]
+        a = mini.greedy_alignment(rows) if len(rows) else np.zeros(0, np.int32)
+        np.testing.assert_array_equal(o["frame_argmax"][off[b]:off[b + 1]], a)
+        H = [mini.frame_entropy(r) for r in rows]
+        np.testing.assert_allclose(o["frame_entropy"][off[b]:off[b + 1]], H, rtol=0, atol=1e-12)
+        y = mini.collapse(a, blank)
+        assert o["draft_full_len"][b] == len(y) and o["draft_len"][b] == min(len(y), cap)
+        n = int(o["draft_len"][b])
+        assert list(o["draft_tokens"][off[b]:off[b] + n]) == y[:n]
+        if len(H) and abs(max(H) - tau_c) > 1e-9:
+            assert bool(g["gate_accept"][b]) == mini.gate(H, tau_c)
+    # stage 2 on its own ragged batch
+    Vl = int(rng.integers(2, 60))
+    K = rng.integers(0, 15, size=B)
+    toff = np.concatenate([[0], np.cumsum(K)]).astype(np.int64)
+    xl = to_storage(rng.normal(size=(int(toff[-1]), Vl)) * 4.0, dtype)
+    ids = rng.integers(0, Vl, size=int(toff[-1])).astype(np.int32)
+    tau_s = float(rng.choice([0.02, 0.1, 0.2, 0.5]))
+    v = ref.verify(xl, Vl, toff, ids, tau_s)
+    gr = ref.greedy_step(xl, Vl) if len(ids) else None
+    xlw = mini.widen(xl).reshape(-1, Vl)
+    for b in range(B):
+        rows, d = xlw[toff[b]:toff[b + 1]], ids[toff[b]:toff[b + 1]]
+        p = mini.token_likelihoods(rows, d)
+        np.testing.assert_allclose(np.exp(v["token_logp"][toff[b]:toff[b + 1]]), p, rtol=1e-12, atol=0)
+        if len(p) == 0 or np.abs(p - tau_s).min() > 1e-9:
+            assert v["accepted_len"][b] == mini.accepted_prefix(p, tau_s)
+        for i, r in enumerate(rows):
+            tok, lp = mini.greedy_token(r)
+            assert gr["next_token"][toff[b] + i] == tok
+            assert abs(gr["next_logp"][toff[b] + i] - lp) < 1e-12
