@@ -47,6 +47,10 @@ def parse_args():
                          "shape at its high-accuracy / high-RTFx operating point")
     ap.add_argument("--e2e-steps", type=int, default=30)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--verify-mode", default="full", choices=["full", "early_exit"],
+                    help="full: ssd_verify reads every row of every verified utterance (the "
+                         "benchmark metric); early_exit: ssd_verify_early_exit in its place, a "
+                         "separate mode whose line says so in config.verify_mode")
     ap.add_argument("--sweep", default=None, metavar="FILE",
                     help="time every point of the throughput sweep (configuration 4) and write one "
                          "JSON line per point to FILE instead of the benchmark line")
@@ -145,7 +149,7 @@ def summarise_clocks(rows, windows, note):
 
 
 # ---- our arm ---------------------------------------------------------------------------------
-def build_sets(w, device, n_sets, batch_lengths=None):
+def build_sets(w, device, n_sets, batch_lengths=None, verify_mode="full"):
     """Input sets and pre-marshalled calls.  The verify logits of a set have one row per draft
     token of the set's own CTC drafts (found by running stage 1 once, untimed).  With
     batch_lengths (a list of per-batch utterance lengths) every set is one of those batches."""
@@ -176,14 +180,30 @@ def build_sets(w, device, n_sets, batch_lengths=None):
         skipped = gate["gate_accept"].cpu().numpy().astype(bool)
         m_active = int(sum(k for k, s in zip(K, skipped) if not s))
         es = 2 if wi.dtype == "bf16" else 4
+        if verify_mode == "early_exit":
+            # the full call first (its decisions are the check), then the early-exit one, whose
+            # rows_read give the bytes this mode really reads
+            ssd.ssd_verify(vb.logits, tok_off, ids, wi.tau_slm, skip=gate["gate_accept"], out=s2)
+            full_acc = s2["accepted_len"].clone()
+            s2 = ssd.alloc_early_exit_outputs(M, B, wi.V_llm, code, device)
+            call_verify = ssd.bind_verify_early_exit(vb.logits, tok_off, ids, wi.tau_slm, s2,
+                                                     skip=gate["gate_accept"])
+            call_verify()
+            torch.cuda.synchronize()
+            assert torch.equal(full_acc, s2["accepted_len"]), "early exit changed a decision"
+            rr = s2["rows_read"]
+            if bool((rr >= 0).all().item()):
+                m_active = int(rr.sum().item())
+        else:
+            call_verify = ssd.bind_verify(vb.logits, tok_off, ids, wi.tau_slm, s2,
+                                          skip=gate["gate_accept"])
         sets.append(dict(
             w=wi, cb=cb, vb=vb, off=off, tok_off=tok_off, ids=ids, s1=s1, gate=gate, s2=s2,
             B=B, N=N, M=M, K=K, m_active=m_active,
             ctc_bytes=N * wi.V_ctc * es, verify_bytes=m_active * wi.V_llm * es,
             call_ctc=ssd.bind_ctc_draft(cb.logits, off, wi.blank_id, wi.max_draft_len, s1),
             call_gate=ssd.bind_entropy_gate(s1["frame_entropy"], off, wi.tau_ctc, gate),
-            call_verify=ssd.bind_verify(vb.logits, tok_off, ids, wi.tau_slm, s2,
-                                        skip=gate["gate_accept"])))
+            call_verify=call_verify))
     return sets
 
 
@@ -222,7 +242,7 @@ def run_ours(args):
         # the paper's batching: a pool of utterances, length-sorted, <= 50,000 frames per batch
         batch_lengths = synth.length_sorted_batches(synth.draw_lengths(w))
         n_sets = 1 if args.ncu_small else len(batch_lengths)
-    sets = build_sets(w, device, n_sets, batch_lengths)
+    sets = build_sets(w, device, n_sets, batch_lengths, args.verify_mode)
     K, W = args.steps, args.warmup
 
     def step(s, o_ctc=None, o_ver=None):
@@ -286,6 +306,8 @@ def run_ours(args):
                                  for i in range(K))
     peak, peak_kind = peaks()
 
+    vkern = "verify_rows_tma" if args.verify_mode == "full" else "verify_rows_ee"
+
     def roof(kernel, nbytes, times_ms):
         avg = statistics.mean(times_ms)
         ach = nbytes / (avg * 1e-3) / 1e9 if avg > 0 else 0.0
@@ -303,7 +325,8 @@ def run_ours(args):
     if rank != 0:
         D.finalize()
         return
-    next_rows = None if args.ncu_small else time_next_rows(sets, device, peak)
+    next_rows = None if (args.ncu_small or args.verify_mode != "full") else \
+        time_next_rows(sets, device, peak)
     s0 = sets[0]
     gate_acc = float(s0["gate"]["gate_accept"].float().mean().item())
     all_acc = s0["s2"]["all_accepted"].cpu().numpy().astype(bool)
@@ -321,6 +344,7 @@ def run_ours(args):
                          % (w.B, len(batch_lengths)),
                          w.t_dist, w.t_lo, w.t_hi, w.V_ctc, w.V_llm, w.max_draft_len, w.dtype),
             "generator": w.variant, "tau_ctc": w.tau_ctc, "tau_slm": w.tau_slm,
+            "verify_mode": args.verify_mode,
             "frames_per_step": s0["N"], "verify_rows_per_step": s0["M"],
             "verify_rows_read_per_step": s0["m_active"],
             "logits_bytes_per_step": int(step_bytes),
@@ -328,12 +352,12 @@ def run_ours(args):
                   "step reads %.2f GB once" % (n_sets, (s0["ctc_bytes"] + s0["M"] * w.V_llm * 2) / 1e9,
                                               step_bytes / 1e9),
             "parallelism": "utterances sharded over %d rank(s), no data-path collective" % world},
-        "gpu_launches": 5 * K,
+        "gpu_launches": (5 if args.verify_mode == "full" else 6) * K,
         # `roofline` is the kernel that holds most of the step's device time
-        "roofline": roof("verify_rows_tma", ver_bytes, t_ver) if sum(t_ver) >= sum(t_ctc)
+        "roofline": roof(vkern, ver_bytes, t_ver) if sum(t_ver) >= sum(t_ctc)
                     else roof("ctc_rows_tma", ctc_bytes, t_ctc),
         "roofline_ctc": roof("ctc_rows_tma", ctc_bytes, t_ctc),
-        "roofline_verify": roof("verify_rows_tma", ver_bytes, t_ver),
+        "roofline_verify": roof(vkern, ver_bytes, t_ver),
         "step_hbm_gbs": round(step_bytes / (ms_max / K * 1e-3) / 1e9, 1),
         "step_frac_of_peak": round(step_bytes / (ms_max / K * 1e-3) / 1e9 / peak, 4),
         "decisions": {"gate_accept_frac": round(gate_acc, 4),
