@@ -25,10 +25,18 @@ struct Launch {
 // the stream is still running, which takes the launch latency of the short per-utterance
 // kernels off the critical path.  A kernel first lets its own successor be scheduled, then
 // waits until every earlier grid has completed and its writes are visible; nothing before
-// pdl_enter() touches global memory.
-__device__ __forceinline__ void pdl_enter() {
+// pdl_enter() / pdl_wait() touches global memory.  The streaming kernels call the two halves
+// apart, with their shared-memory set-up in between, so that the set-up (and the cold
+// instruction fetches that come with it) overlaps the predecessor's tail.
+__device__ __forceinline__ void pdl_launch_dependents() {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void pdl_wait() {
     asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+__device__ __forceinline__ void pdl_enter() {
+    pdl_launch_dependents();
+    pdl_wait();
 }
 
 template <typename... KArgs, typename... Args>

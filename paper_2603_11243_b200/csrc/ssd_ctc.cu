@@ -309,10 +309,12 @@ template <typename T, int G>
 __global__ void __launch_bounds__(768, 1) ctc_rows_tma(const CtcParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     constexpr int ES = Elem<T>::kBytes;
-    pdl_enter();
+    pdl_launch_dependents();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int W = p.warps, S = p.stages, R = p.rows_per_tile;
-    const int64_t gw = (int64_t)blockIdx.x * W + warp, GW = (int64_t)gridDim.x * W;
+    // Tile j goes to CTA j mod grid, and within the CTA to warp (j / grid) mod W: every CTA
+    // gets the same number of tiles (give or take one) whatever the size of the matrix.
+    const int64_t gw = (int64_t)blockIdx.x + (int64_t)gridDim.x * warp, GW = (int64_t)gridDim.x * W;
     const int64_t my_tiles = gw < p.num_tiles ? (p.num_tiles - gw + GW - 1) / GW : 0;
     if (my_tiles == 0) return;
 
@@ -392,6 +394,7 @@ __global__ void __launch_bounds__(768, 1) ctc_rows_tma(const CtcParams p) {
         }
     };
 
+    pdl_wait();
     const int prologue = (int)min((int64_t)S, my_tiles);
     for (int k = 0; k < prologue; ++k) issue(k, k);
 
@@ -711,7 +714,7 @@ int launch_ctc_rows(const void *logits, ssd_dtype dtype, int V, int64_t ld, int6
         p.num_tiles = (N + R - 1) / R;
         const size_t smem = (size_t)((warps * stages * 8 + 127) & ~127) +
                             (size_t)warps * stages * p.stage_stride;
-        int64_t ctas = (p.num_tiles + warps - 1) / warps;
+        int64_t ctas = p.num_tiles;
         const int max_ctas = (o && o->ctas > 0) ? o->ctas : sm_count();
         if (ctas > max_ctas) ctas = max_ctas;
         void (*kern)(const CtcParams) = nullptr;

@@ -50,7 +50,7 @@ template <typename T, int kF, bool kArg>
 __global__ void __launch_bounds__(544, 1) verify_rows_tma(const VerifyParams p) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     constexpr int ES = Elem<T>::kBytes, EPC = Elem<T>::kPerChunk;
-    pdl_enter();
+    pdl_launch_dependents();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int S = p.stages, CW = p.warps;
     // layout: full[S] | empty[S] | desc[S] | offsets cache | stages
@@ -70,6 +70,7 @@ __global__ void __launch_bounds__(544, 1) verify_rows_tma(const VerifyParams p) 
         for (int s = 0; s < S; ++s) { mbar_init(full0 + s * 8, 1); mbar_init(empty0 + s * 8, CW); }
         mbar_init_fence();
     }
+    pdl_wait();
     if (cache_off)
         for (int i = threadIdx.x; i <= p.B; i += blockDim.x) off_cache[i] = p.tok_off[i];
     __syncthreads();
@@ -270,9 +271,14 @@ __global__ void __launch_bounds__(kFinishThreads) verify_finish_kernel(
     __shared__ int first_reject;
     __shared__ unsigned flags;
     pdl_enter();
+    // The kernel is a chain of dependent memory round trips, so the loads of each level are
+    // issued together: offsets, skip flag and error word; then a row's draft id and its
+    // partials; then the draft token's logit.
     const int b = blockIdx.x, tid = threadIdx.x;
     const int64_t i0 = tok_off[b], i1 = tok_off[b + 1];
-    const uint32_t internal = (*err_word == epoch) ? (uint32_t)SSD_UTT_INTERNAL : 0u;
+    const unsigned long long err = *err_word;
+    const bool skipped = skip != nullptr && skip[b] != 0;
+    const uint32_t internal = (err == epoch) ? (uint32_t)SSD_UTT_INTERNAL : 0u;
     if (i0 < 0 || i1 < i0 || i1 > M) {
         if (tid == 0) {
             accepted_len[b] = 0; all_accepted[b] = 0;
@@ -282,7 +288,7 @@ __global__ void __launch_bounds__(kFinishThreads) verify_finish_kernel(
     }
     const int64_t K64 = i1 - i0;
     const int K = K64 > 0x7fffffff ? 0x7fffffff : (int)K64;
-    if (skip && skip[b]) {
+    if (skipped) {
         if (tid == 0) { accepted_len[b] = K; all_accepted[b] = 1; utt_status[b] = internal; }
         return;
     }
@@ -292,20 +298,26 @@ __global__ void __launch_bounds__(kFinishThreads) verify_finish_kernel(
     int myfirst = K;
     for (int i = tid; i < K; i += blockDim.x) {
         const int64_t r = i0 + i;
-        // P (reference, sum) pairs of this row; read two at a time where P is even
+        const int id = draft_ids[r];
+        const bool id_ok = id >= 0 && id < V;
+        // P (reference, sum) pairs of this row; up to 16 are read two at a time into registers
         const float2 *pp = partials + r * P;
         float Mx = kNegInit, S = 0.f;
-        if ((P & 1) == 0) {
+        float x = 0.f;
+        if ((P & 1) == 0 && P <= 16) {
             const float4 *p4 = reinterpret_cast<const float4 *>(pp);
-            for (int q = 0; q < P / 2; ++q) {
-                const float4 v = p4[q];
-                Mx = fmaxf(Mx, fmaxf(v.x, v.z));
-            }
-            for (int q = 0; q < P / 2; ++q) {
-                const float4 v = p4[q];
-                S += v.y * ex2((v.x - Mx) * kLog2e) + v.w * ex2((v.z - Mx) * kLog2e);
-            }
+            float4 v[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                v[q] = q < P / 2 ? p4[q] : make_float4(kNegInit, 0.f, kNegInit, 0.f);
+            if (id_ok) x = Elem<T>::load(logits + (r * ld + id) * ES);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) Mx = fmaxf(Mx, fmaxf(v[q].x, v[q].z));
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                S += v[q].y * ex2((v[q].x - Mx) * kLog2e) + v[q].w * ex2((v[q].z - Mx) * kLog2e);
         } else {
+            if (id_ok) x = Elem<T>::load(logits + (r * ld + id) * ES);
             for (int q = 0; q < P; ++q) Mx = fmaxf(Mx, pp[q].x);
             for (int q = 0; q < P; ++q) {
                 const float2 v = pp[q];
@@ -315,15 +327,13 @@ __global__ void __launch_bounds__(kFinishThreads) verify_finish_kernel(
         const float lnS = logf(S);
         const float lse = Mx + lnS;
         if (!(fabsf(lse) < INFINITY)) myflags |= SSD_UTT_NONFINITE;
-        const int id = draft_ids[r];
         float logp;
         bool reject;
-        if (id < 0 || id >= V) {
+        if (!id_ok) {
             myflags |= SSD_UTT_BAD_DRAFT_ID;
             logp = -INFINITY;
             reject = true;
         } else {
-            const float x = Elem<T>::load(logits + (r * ld + id) * ES);
             logp = (x - Mx) - lnS;      // not x - lse: keeps its accuracy when |x| is large
             reject = reject_none ? false : !(logp > log_tau);   // p <= tau; NaN rejects
         }

@@ -88,7 +88,7 @@ template <typename T, int kF>
 __global__ void __launch_bounds__(544, 1) verify_rows_ee(const EeParams p) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     constexpr int ES = Elem<T>::kBytes, EPC = Elem<T>::kPerChunk;
-    pdl_enter();
+    pdl_launch_dependents();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int S = p.stages, CW = p.warps, NR = 2 * S;
     // layout: full[S] | empty[S] | desc[S] | pending[S] | rowmeta[NR] | sx[NR] | spart[NR*CW] |
@@ -119,6 +119,7 @@ __global__ void __launch_bounds__(544, 1) verify_rows_ee(const EeParams p) {
         }
         mbar_init_fence();
     }
+    pdl_wait();
     if (cache_off)
         for (int i = threadIdx.x; i <= p.B; i += blockDim.x) off_cache[i] = p.tok_off[i];
     __syncthreads();
