@@ -536,15 +536,16 @@ __global__ void __launch_bounds__(kUttThreads) collapse_kernel(
     for (int64_t tile = 0; tile < T; tile += blockDim.x, buf ^= 1) {
         const int64_t t = tile + tid;
         const bool valid = t < T;
-        int a = blank_id;
+        int a = blank_id, prev0 = -1;
         float h = 0.f;
         if (valid) {
             a = frame_argmax[t0 + t];
             h = frame_entropy[t0 + t];
+            if (lane == 0 && t > 0) prev0 = frame_argmax[t0 + t - 1];   // issued with the others
         }
         // the previous frame's symbol: the neighbouring lane has it, except for lane 0
         int prev = __shfl_up_sync(0xffffffffu, a, 1);
-        if (lane == 0) prev = (valid && t > 0) ? frame_argmax[t0 + t - 1] : -1;
+        if (lane == 0) prev = prev0;
         if (valid) {
             if (h != h) {
                 myflags |= (__float_as_uint(h) == kNanInternal) ? SSD_UTT_INTERNAL : SSD_UTT_NONFINITE;
