@@ -33,7 +33,8 @@ KERNEL_EVENT_EVERY = 5          # N_SETS and this are coprime: every input set g
 N_SETS = 3                      # distinct input batches rotated through, so no step finds its
                                 # inputs in the 126 MB L2
 TRAFFIC_FILE = os.path.join(ROOT, "paper_2603_11243_b200", "ncu_traffic.json")
-KERNEL_SOURCES = ["ssd_common.cuh", "ssd_stream.cuh", "ssd_ctc.cu", "ssd_verify.cu", "ssd_api.cu"]
+KERNEL_SOURCES = ["ssd_common.cuh", "ssd_stream.cuh", "ssd_ranges.cuh", "ssd_ctc.cu", "ssd_verify.cu",
+                  "ssd_api.cu"]
 
 
 def parse_args():

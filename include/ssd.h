@@ -316,6 +316,38 @@ int32_t ssd_verify_static(const void *logits, ssd_dtype dtype, int32_t V, int64_
                           int32_t *accepted_len, uint8_t *all_accepted, uint32_t *utt_status,
                           void *stream, const ssd_launch_opts *opts);
 
+/*
+ * Read-span hooks.  The paper has no counterpart: these are test hooks of this library, host
+ * only (no GPU, no stream; base_addr is an integer that is never dereferenced).
+ *
+ * The bulk-copy kernels fetch 16-byte-aligned ranges, while rows of logits may start anywhere a
+ * whole element can (odd vocabulary sizes, column slices).  These functions replay on the host
+ * the very address arithmetic those kernels use (one shared header) for a matrix that would
+ * start at base_addr, over all of its tiles (ssd_ctc_draft) or rows, column spans and stage
+ * parts (ssd_verify, whose streaming kernel ssd_greedy_step shares), and report
+ *   lo, hi   the lowest address that would be read and one past the highest
+ *   faults   how many tiles / rows break a rule: a read outside the matrix (outside the row,
+ *            for ssd_verify), a bulk copy off a 16-byte boundary or larger than its stage, or
+ *            reads that do not cover the tile's / row's bytes exactly once
+ *   kernel   2: the bulk-copy kernel would run; 1: the plain-load kernel, which indexes
+ *            elements one by one (lo, hi are then the matrix's own extent)
+ * so a caller -- the tests do -- can assert faults == 0, lo >= base_addr and
+ * hi <= base_addr + ((rows - 1) * ld + V) * element size for any shape and misalignment.
+ * Errors: SSD_ERR_NULL, SSD_ERR_ARG, SSD_ERR_DTYPE, SSD_ERR_ALIGN (base_addr not a multiple of
+ * the element size).
+ */
+typedef struct ssd_read_span {
+    uint64_t lo, hi;
+    int64_t faults;
+    int32_t kernel;
+    int32_t reserved;
+} ssd_read_span;
+int32_t ssd_ctc_draft_read_span(uint64_t base_addr, ssd_dtype dtype, int32_t V, int64_t ld,
+                                int64_t N, const ssd_launch_opts *opts, ssd_read_span *out);
+int32_t ssd_verify_read_span(uint64_t base_addr, ssd_dtype dtype, int32_t V, int64_t ld,
+                             int64_t M, int32_t B, const ssd_launch_opts *opts,
+                             ssd_read_span *out);
+
 #ifdef __cplusplus
 }
 #endif

@@ -72,6 +72,10 @@ def lib():
         L.ssd_verify_early_exit.restype = i32
         L.ssd_verify_early_exit.argtypes = [vp, C.c_int, i32, i64, vp, vp, i32, i64, C.c_float, vp,
                                             vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp, vp]
+        for f in (L.ssd_ctc_draft_read_span, L.ssd_verify_read_span):
+            f.restype = i32
+        L.ssd_ctc_draft_read_span.argtypes = [C.c_uint64, C.c_int, i32, i64, i64, vp, vp]
+        L.ssd_verify_read_span.argtypes = [C.c_uint64, C.c_int, i32, i64, i64, i32, vp, vp]
         L.ssd_threshold_sweep.restype = i32
         L.ssd_threshold_sweep.argtypes = [vp, vp, vp, i32, i64, vp, vp, i32, vp, vp, vp, vp, vp]
         L.ssd_assemble.restype = i32
@@ -121,6 +125,34 @@ def ssd_ctc_draft_workspace_bytes(B, N, V, dtype_code, opts=None) -> int:
 
 def ssd_verify_workspace_bytes(B, M, V, dtype_code, opts=None) -> int:
     return int(lib().ssd_verify_workspace_bytes(B, M, V, dtype_code, _opts(opts)))
+
+
+class ReadSpan(C.Structure):
+    """Mirror of ssd_read_span (include/ssd.h)."""
+    _fields_ = [("lo", C.c_uint64), ("hi", C.c_uint64), ("faults", C.c_int64),
+                ("kernel", C.c_int32), ("reserved", C.c_int32)]
+
+
+def ssd_ctc_draft_read_span(base_addr: int, dtype_code: int, V: int, ld: int, N: int,
+                            opts: Optional[LaunchOpts] = None) -> ReadSpan:
+    """Host-only: the addresses ssd_ctc_draft's streaming kernel would read (see ssd.h)."""
+    out = ReadSpan()
+    rc = lib().ssd_ctc_draft_read_span(base_addr, dtype_code, V, ld, N, _opts(opts),
+                                       C.cast(C.pointer(out), C.c_void_p))
+    if rc != OK:
+        raise SsdError(rc, "ssd_ctc_draft_read_span")
+    return out
+
+
+def ssd_verify_read_span(base_addr: int, dtype_code: int, V: int, ld: int, M: int, B: int = 1,
+                         opts: Optional[LaunchOpts] = None) -> ReadSpan:
+    """Host-only: the addresses ssd_verify's streaming kernel would read (see ssd.h)."""
+    out = ReadSpan()
+    rc = lib().ssd_verify_read_span(base_addr, dtype_code, V, ld, M, B, _opts(opts),
+                                    C.cast(C.pointer(out), C.c_void_p))
+    if rc != OK:
+        raise SsdError(rc, "ssd_verify_read_span")
+    return out
 
 
 def alloc_ctc_outputs(N: int, B: int, device, logprob_ld: int = 0) -> Dict[str, torch.Tensor]:

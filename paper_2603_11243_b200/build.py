@@ -6,7 +6,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libssd.so")
-SOURCES = ["ssd_api.cu", "ssd_ctc.cu", "ssd_verify.cu", "ssd_verify_static.cu", "ssd_decide.cu", "ssd_verify_ee.cu"]
+SOURCES = ["ssd_api.cu", "ssd_ctc.cu", "ssd_verify.cu", "ssd_verify_static.cu", "ssd_decide.cu", "ssd_verify_ee.cu",
+           "ssd_readspan.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--use_fast_math=false", "-Xcompiler", "-fPIC", "-shared", "-cudart", "shared"]
 

@@ -334,6 +334,16 @@ int launch_gate(const float *frame_entropy, const int64_t *frame_off, int B, int
                 float tau, uint8_t *gate_accept, float *max_entropy, int32_t *argmax_frame,
                 cudaStream_t stream);
 
+struct CtcPlan {
+    int kernel;          // 1 plain loads, 2 bulk-copy tiles
+    int lanes_per_row;   // G
+    int rows_per_tile;   // R
+    int warps, stages, stage_stride;
+    int64_t num_tiles;
+};
+int plan_ctc(ssd_dtype dtype, int V, int64_t ld, int64_t N, const ssd_launch_opts *opts,
+             CtcPlan *plan);
+
 struct VerifyPlan {
     int kernel;        // 1 plain loads, 2 bulk-copy pipeline
     int ctas;

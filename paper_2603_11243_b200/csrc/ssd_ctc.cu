@@ -12,6 +12,7 @@
 #include <math.h>
 
 #include "ssd_common.cuh"
+#include "ssd_ranges.cuh"
 
 namespace ssd {
 
@@ -330,64 +331,37 @@ __global__ void __launch_bounds__(768, 1) ctc_rows_tma(const CtcParams p) {
     __syncwarp();
 
     const uintptr_t base = reinterpret_cast<uintptr_t>(p.logits);
-    const uintptr_t lo_bound = base, hi_bound = base + (uintptr_t)p.total_bytes;
     const int64_t row_pitch = p.ld * ES;
 
     // Brings tile k of this warp into stage s.  The tile's rows are one contiguous byte range
     // (padding between rows included); the 16-byte-aligned superset of the range is fetched with
-    // one bulk copy.  Only for the first and the last tile of the matrix may that superset leave
-    // the matrix: there the bulk copy is shortened and the few elements outside it are fetched
-    // with plain loads.  Bytes of neighbouring rows that come along are never looked at.
-    const int64_t tile_bytes = (int64_t)(R - 1) * row_pitch + (int64_t)p.V * ES;
+    // one bulk copy, except where that superset would leave the matrix (near its two ends):
+    // there the copy is one chunk shorter and the few elements outside it are fetched with
+    // plain loads.  Bytes of neighbouring rows that come along are never looked at.
     auto issue = [&](int64_t k, int s) {
-        const int64_t tile = gw + k * GW;
-        const uintptr_t gstart = base + (uintptr_t)(tile * R * row_pitch);
+        const ranges::TileReads t = ranges::tile_reads(base, p.total_bytes, row_pitch,
+                                                       (int64_t)p.V * ES, p.N, R, gw + k * GW);
         const uint32_t bar = bar0 + s * 8;
-        if (tile != 0 && tile != p.num_tiles - 1) {
-            if (lane == 0) {
-                const uintptr_t f0 = gstart & ~(uintptr_t)15;
-                const uint32_t bytes = (uint32_t)(((gstart + tile_bytes + 15) & ~(uintptr_t)15) - f0);
-                fence_proxy_async();
-                mbar_arrive_expect_tx(bar, bytes);
-                bulk_g2s(stage0 + (uint32_t)s * p.stage_stride, reinterpret_cast<const void *>(f0),
-                         bytes, bar);
-            }
-            return;
-        }
-        const int nrows = (int)min((int64_t)R, p.N - tile * R);
-        const uintptr_t gend = gstart + (uintptr_t)((nrows - 1) * row_pitch + (int64_t)p.V * ES);
-        const uintptr_t f0 = gstart & ~(uintptr_t)15;
-        const uintptr_t c1 = (gend + 15) & ~(uintptr_t)15;
-        const uintptr_t bulk_lo = f0 >= lo_bound ? f0 : f0 + 16;
-        const uintptr_t bulk_hi = c1 <= hi_bound ? c1 : c1 - 16;
-        const bool has_bulk = bulk_hi > bulk_lo;
         unsigned char *dst = stage0_ptr + (size_t)s * p.stage_stride;
-        if (!has_bulk || bulk_lo > gstart || bulk_hi < gend) {
-            const uintptr_t h_end = has_bulk ? min(bulk_lo, gend) : gend;
-            for (uintptr_t a = gstart + (uintptr_t)lane * ES; a < h_end; a += 32 * ES) {
-                if (ES == 4) *reinterpret_cast<uint32_t *>(dst + (a - f0)) =
-                        *reinterpret_cast<const uint32_t *>(a);
-                else *reinterpret_cast<uint16_t *>(dst + (a - f0)) =
-                        *reinterpret_cast<const uint16_t *>(a);
-            }
-            if (has_bulk) {
-                for (uintptr_t a = max(bulk_hi, gstart) + (uintptr_t)lane * ES; a < gend;
-                     a += 32 * ES) {
-                    if (ES == 4) *reinterpret_cast<uint32_t *>(dst + (a - f0)) =
+        if (t.head_hi > t.head_lo || t.tail_hi > t.tail_lo) {
+            for (int side = 0; side < 2; ++side) {
+                const uintptr_t lo = side ? t.tail_lo : t.head_lo, hi = side ? t.tail_hi : t.head_hi;
+                for (uintptr_t a = lo + (uintptr_t)lane * ES; a < hi; a += 32 * ES) {
+                    if (ES == 4) *reinterpret_cast<uint32_t *>(dst + (a - t.f0)) =
                             *reinterpret_cast<const uint32_t *>(a);
-                    else *reinterpret_cast<uint16_t *>(dst + (a - f0)) =
+                    else *reinterpret_cast<uint16_t *>(dst + (a - t.f0)) =
                             *reinterpret_cast<const uint16_t *>(a);
                 }
             }
             __syncwarp();
         }
         if (lane == 0) {
-            if (has_bulk) {
-                const uint32_t bytes = (uint32_t)(bulk_hi - bulk_lo);
+            if (t.bulk_hi > t.bulk_lo) {
+                const uint32_t bytes = (uint32_t)(t.bulk_hi - t.bulk_lo);
                 fence_proxy_async();
                 mbar_arrive_expect_tx(bar, bytes);
-                bulk_g2s(stage0 + (uint32_t)s * p.stage_stride + (uint32_t)(bulk_lo - f0),
-                         reinterpret_cast<const void *>(bulk_lo), bytes, bar);
+                bulk_g2s(stage0 + (uint32_t)s * p.stage_stride + (uint32_t)(t.bulk_lo - t.f0),
+                         reinterpret_cast<const void *>(t.bulk_lo), bytes, bar);
             } else {
                 mbar_arrive(bar);
             }
@@ -651,24 +625,12 @@ unsigned long long next_epoch() {
     return 0x55D0000000000000ull | (c & 0x0000ffffffffffffull);
 }
 
-int launch_ctc_rows(const void *logits, ssd_dtype dtype, int V, int64_t ld, int64_t N,
-                    const int64_t *frame_off, int B, float *frame_entropy, int32_t *frame_argmax,
-                    float *frame_lse, float *frame_logprob, uint32_t *utt_status,
-                    const Launch &L) {
-    (void)frame_off; (void)B; (void)utt_status;
-    if (N == 0) return SSD_OK;
-    const ssd_launch_opts *o = L.opts;
+// Kernel and launch shape of the frame-statistics pass for these sizes.
+// G lanes share a row (so that a lane walks about 8..18 chunks of 16 bytes), a warp works on
+// 32/G rows at a time, and a tile is a whole number of such row groups of about 8 KB.
+int plan_ctc(ssd_dtype dtype, int V, int64_t ld, int64_t N, const ssd_launch_opts *o, CtcPlan *plan) {
     const int es = dtype == SSD_F32 ? 4 : 2;
-    CtcParams p{};
-    p.logits = static_cast<const char *>(logits);
-    p.V = V; p.ld = ld; p.N = N;
-    p.total_bytes = (N - 1) * ld * es + (int64_t)V * es;
-    p.frame_entropy = frame_entropy; p.frame_argmax = frame_argmax; p.frame_lse = frame_lse;
-    p.frame_logprob = frame_logprob;
-
-    // ---- choose the kernel and its shape ----
-    // G lanes share a row (so that a lane walks about 8..18 chunks of 16 bytes), a warp works
-    // on 32/G rows at a time, and a tile is a whole number of such row groups of about 8 KB.
+    CtcPlan pl{};
     int kernel = o ? o->kernel : 0;
     const int64_t row_pitch = ld * es;
     const int64_t row_bytes = (int64_t)V * es;
@@ -704,6 +666,33 @@ int launch_ctc_rows(const void *logits, ssd_dtype dtype, int V, int64_t ld, int6
     } else {
         kernel = 2;
     }
+    pl.kernel = kernel; pl.lanes_per_row = G; pl.rows_per_tile = R; pl.warps = warps;
+    pl.stages = stages; pl.stage_stride = (int)stage_stride;
+    pl.num_tiles = kernel == 2 ? (N + R - 1) / R : 0;
+    *plan = pl;
+    return SSD_OK;
+}
+
+int launch_ctc_rows(const void *logits, ssd_dtype dtype, int V, int64_t ld, int64_t N,
+                    const int64_t *frame_off, int B, float *frame_entropy, int32_t *frame_argmax,
+                    float *frame_lse, float *frame_logprob, uint32_t *utt_status,
+                    const Launch &L) {
+    (void)frame_off; (void)B; (void)utt_status;
+    if (N == 0) return SSD_OK;
+    const ssd_launch_opts *o = L.opts;
+    const int es = dtype == SSD_F32 ? 4 : 2;
+    CtcParams p{};
+    p.logits = static_cast<const char *>(logits);
+    p.V = V; p.ld = ld; p.N = N;
+    p.total_bytes = (N - 1) * ld * es + (int64_t)V * es;
+    p.frame_entropy = frame_entropy; p.frame_argmax = frame_argmax; p.frame_lse = frame_lse;
+    p.frame_logprob = frame_logprob;
+    CtcPlan plan;
+    const int prc = plan_ctc(dtype, V, ld, N, o, &plan);
+    if (prc != SSD_OK) return prc;
+    const int kernel = plan.kernel, G = plan.lanes_per_row, R = plan.rows_per_tile;
+    const int warps = plan.warps, stages = plan.stages;
+    const int64_t stage_stride = plan.stage_stride;
     cudaError_t e;
     if (o && o->ev_begin) {
         e = cudaEventRecord(static_cast<cudaEvent_t>(o->ev_begin), L.stream);

@@ -17,6 +17,7 @@
 #include <math.h>
 
 #include "ssd_common.cuh"
+#include "ssd_ranges.cuh"
 #include "ssd_stream.cuh"
 
 namespace ssd {
@@ -100,29 +101,23 @@ __global__ void __launch_bounds__(544, 1) verify_rows_tma(const VerifyParams p) 
                 todo &= todo - 1;
                 const int64_t row = __shfl_sync(0xffffffffu, my_row, src);
                 const int sp = (int)(__shfl_sync(0xffffffffu, mine, src) - row * p.split);
-                const uintptr_t g0 = reinterpret_cast<uintptr_t>(p.logits) +
-                                     (uintptr_t)(row * p.ld * ES);
-                const uintptr_t g1 = g0 + (uintptr_t)row_bytes;
-                const uintptr_t f0 = g0 & ~(uintptr_t)15;
-                const int row_chunks = (int)((((g1 + 15) & ~(uintptr_t)15) - f0) >> 4);
-                const int cps = (row_chunks + p.split - 1) / p.split;
-                const int sc0 = min(row_chunks, sp * cps), sc1 = min(row_chunks, sc0 + cps);
-                const int span = sc1 - sc0;
-                const int parts = span > 0 ? (span + max_chunks - 1) / max_chunks : 1;
-                const int per_part = span > 0 ? (span + parts - 1) / parts : 0;
+                const ranges::RowGeom geom = ranges::row_geom(
+                    reinterpret_cast<uintptr_t>(p.logits), row, p.ld * ES, row_bytes);
+                const uintptr_t g0 = geom.g0, g1 = geom.g1, f0 = geom.f0;
+                const ranges::SpanCut cut = ranges::span_cut(geom.row_chunks, p.split, sp, max_chunks);
+                const int sc1 = cut.sc1, parts = cut.parts, per_part = cut.per_part;
                 const int64_t slot = row * p.partials_per_row + (int64_t)sp * CW;
-                const bool head_ragged = f0 != g0, tail_ragged = (g1 & 15) != 0;
                 for (int part = 0; part < parts; ++part) {
                     if (!mbar_wait_bounded(empty0 + s * 8, ph ^ 1u)) { failed = true; break; }
-                    const int pc0 = sc0 + part * per_part;
+                    const int pc0 = cut.sc0 + part * per_part;
                     const int pc1 = min(sc1, pc0 + per_part);
                     // chunks that are only partly inside the row (row start / end not on a
                     // 16-byte boundary) are filled here with plain loads and -inf padding; the
                     // bulk copy takes the fully valid chunks only, so it never leaves the row.
-                    int b0 = pc0, b1 = pc1;
+                    const ranges::PartReads pr = ranges::part_reads(geom, pc0, pc1);
+                    const int b0 = pr.b0, b1 = pr.b1;
                     unsigned char *dst = stage0_ptr + (size_t)s * p.stage_bytes;
-                    if (head_ragged && pc1 > pc0 && pc0 == 0) {
-                        b0 = 1;
+                    if (pr.head_plain) {
                         if (lane < EPC) {
                             const uintptr_t a = f0 + (uintptr_t)lane * ES;
                             const bool ok = a >= g0 && a < g1;
@@ -132,9 +127,7 @@ __global__ void __launch_bounds__(544, 1) verify_rows_tma(const VerifyParams p) 
                                 ok ? *reinterpret_cast<const uint16_t *>(a) : (uint16_t)0xff80u;
                         }
                     }
-                    if (tail_ragged && pc1 > pc0 && pc1 == row_chunks &&
-                        !(b0 == 1 && row_chunks == 1)) {
-                        b1 = pc1 - 1;
+                    if (pr.tail_plain) {
                         if (lane < EPC) {
                             const uintptr_t a = f0 + (uintptr_t)(pc1 - 1) * 16 + (uintptr_t)lane * ES;
                             const bool ok = a >= g0 && a < g1;

@@ -16,6 +16,7 @@
 #include <math.h>
 
 #include "ssd_common.cuh"
+#include "ssd_ranges.cuh"
 #include "ssd_stream.cuh"
 
 namespace ssd {
@@ -220,14 +221,12 @@ __global__ void __launch_bounds__(544, 1) verify_rows_ee(const EeParams p) {
                 // a smaller rejected position already known: the row cannot matter
                 if (pos > fr) continue;
                 const bool id_ok = id >= 0 && id < p.V;
-                const uintptr_t g0 = reinterpret_cast<uintptr_t>(p.logits) +
-                                     (uintptr_t)(row * p.ld * ES);
-                const uintptr_t g1 = g0 + (uintptr_t)row_bytes;
-                const uintptr_t f0 = g0 & ~(uintptr_t)15;
-                const int row_chunks = (int)((((g1 + 15) & ~(uintptr_t)15) - f0) >> 4);
-                const int parts = (row_chunks + max_chunks - 1) / max_chunks;
-                const int per_part = (row_chunks + parts - 1) / parts;
-                const bool head_ragged = f0 != g0, tail_ragged = (g1 & 15) != 0;
+                const ranges::RowGeom geom = ranges::row_geom(
+                    reinterpret_cast<uintptr_t>(p.logits), row, p.ld * ES, row_bytes);
+                const uintptr_t g0 = geom.g0, g1 = geom.g1, f0 = geom.f0;
+                const int row_chunks = geom.row_chunks;
+                const ranges::SpanCut cut = ranges::span_cut(row_chunks, 1, 0, max_chunks);
+                const int parts = cut.parts, per_part = cut.per_part;
                 const int64_t id_byte = id_ok ? (int64_t)(g0 - f0) + (int64_t)id * ES : -1;
                 const int rslot = rowseq % NR;
                 ++rowseq;
@@ -241,10 +240,10 @@ __global__ void __launch_bounds__(544, 1) verify_rows_ee(const EeParams p) {
                     finalize(s);
                     const int pc0 = part * per_part;
                     const int pc1 = min(row_chunks, pc0 + per_part);
-                    int b0 = pc0, b1 = pc1;
+                    const ranges::PartReads pr = ranges::part_reads(geom, pc0, pc1);
+                    const int b0 = pr.b0, b1 = pr.b1;
                     unsigned char *dst = stage0_ptr + (size_t)s * p.stage_bytes;
-                    if (head_ragged && pc1 > pc0 && pc0 == 0) {
-                        b0 = 1;
+                    if (pr.head_plain) {
                         if (lane < EPC) {
                             const uintptr_t a = f0 + (uintptr_t)lane * ES;
                             const bool ok = a >= g0 && a < g1;
@@ -254,9 +253,7 @@ __global__ void __launch_bounds__(544, 1) verify_rows_ee(const EeParams p) {
                                 ok ? *reinterpret_cast<const uint16_t *>(a) : (uint16_t)0xff80u;
                         }
                     }
-                    if (tail_ragged && pc1 > pc0 && pc1 == row_chunks &&
-                        !(b0 == 1 && row_chunks == 1)) {
-                        b1 = pc1 - 1;
+                    if (pr.tail_plain) {
                         if (lane < EPC) {
                             const uintptr_t a = f0 + (uintptr_t)(pc1 - 1) * 16 + (uintptr_t)lane * ES;
                             const bool ok = a >= g0 && a < g1;

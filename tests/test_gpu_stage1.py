@@ -94,6 +94,22 @@ def test_odd_vocabulary_sizes(cuda_device, kernel, dtype, V):
     H.compare_stage1(out, gate, orc, cb.frame_off.numpy(), 0.31, require_all_margins=False)
 
 
+@pytest.mark.parametrize("V,T", [(1, [4096, 4096, 1]), (3, [1360, 1360, 1]), (3, [2000, 720, 2]),
+                                 (5, [816, 816, 816, 1])])
+def test_last_tile_of_a_few_bytes(cuda_device, V, T):
+    """Tiny vocabularies make tiles of thousands of rows; a matrix that ends with a tile of one
+    or two rows (fewer than 16 bytes) has its second-to-last tile fetched with a shortened bulk
+    copy plus plain loads.  (That no read leaves the matrix is checked on the host, in
+    test_read_span.py; this checks the values.)"""
+    w = synth.scaled(synth.CONFIGS[1], B=len(T), V_ctc=V, dtype="bf16", variant="literal",
+                     tau_ctc=0.31, seed=300 + V, max_draft_len=50)
+    cb = synth.make_ctc_batch(w, "cpu", T)
+    x = cb.logits.to(cuda_device)
+    out, gate = run_stage1(x, cb.frame_off, V, 0, 50, 0.31, KERNELS["tma"])
+    orc = H.oracle_stage1(H.storage_numpy(cb.logits), V, cb.frame_off.numpy(), 0, 50, 0.31)
+    H.compare_stage1(out, gate, orc, cb.frame_off.numpy(), 0.31, require_all_margins=False)
+
+
 @pytest.mark.parametrize("kernel", KERNELS.values(), ids=KERNELS.keys())
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_padded_rows_and_misaligned_base(cuda_device, kernel, dtype):
