@@ -1,4 +1,5 @@
-"""Parity at the full sizes of the benchmark configurations, in the launch configuration
+"""Parity at the full sizes of the benchmark configurations (and of sampled points of the
+throughput sweep), in the launch configuration
 bench.py times (default options, inputs generated on the device): every output of
 configuration 1 against the oracle; for configurations 2 and 3 (10 and 46 GB of verify logits)
 the GPU computes everything and the oracle recomputes a sample of utterances, chosen to include
@@ -154,3 +155,18 @@ def test_paper_shape_batches(cuda_device, cfg):
             np.testing.assert_array_equal(ga, cb.confident.numpy())
         sample = pick(np.array(lengths), ga, min(5, len(lengths)))
         check_sample(wb, cb, vb, s1, gate, s2, sample)
+
+
+@pytest.mark.parametrize("B,V,dtype", [(1, 100352, "bf16"), (8, 152064, "f32"), (64, 32000, "bf16"),
+                                       (256, 49152, "f32")])
+def test_sweep_points_sampled(cuda_device, B, V, dtype):
+    """Points of the throughput sweep (configuration 4) at their full size, spanning its batch
+    sizes, vocabularies and both dtypes; few rows (B = 1, 8) take the column-span path of
+    ssd_verify.  The GPU computes everything, the oracle recomputes a sample of utterances."""
+    w = synth.sweep_point(B, V, dtype)
+    cb, vb, s1, gate, s2, K = run_path(w, cuda_device)
+    global_properties(w, cb, vb, s1, gate, s2, K)
+    sample = sorted({0, B - 1, B // 2})
+    check_sample(w, cb, vb, s1, gate, s2, sample)
+    del cb, vb, s1, gate, s2
+    torch.cuda.empty_cache()
