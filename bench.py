@@ -58,6 +58,9 @@ def parse_args():
     ap.add_argument("--sweep-filter", default="", help="only points whose name contains this")
     ap.add_argument("--ncu-small", action="store_true",
                     help="profiling aid: one input set, no end-to-end leg, no CPU baseline")
+    ap.add_argument("--ncu-stage1", action="store_true",
+                    help="profiling aid: only the CTC batch of --config (a fraction of a GB even "
+                         "where the whole step holds tens), ssd_ctc_draft three times, no timing")
     return ap.parse_args()
 
 
@@ -709,10 +712,32 @@ def run_sweep(args):
                     print(json.dumps(line), flush=True)
 
 
+def run_stage1_only(args):
+    """Stage 1 alone on one configuration's CTC batch, for a profiler capture of its kernels."""
+    import torch
+    from paper_2603_11243_b200 import binding as ssd
+    from paper_2603_11243_b200 import build as lib_build
+    from paper_2603_11243_b200 import synth
+    lib_build.build()
+    device = torch.device("cuda", 0)
+    w = synth.CONFIGS[args.config]
+    cb = synth.make_ctc_batch(w, device)
+    off = cb.frame_off.to(device)
+    out = ssd.alloc_ctc_outputs(cb.logits.shape[0], w.B, device)
+    for _ in range(3):
+        ssd.ssd_ctc_draft(cb.logits, off, w.blank_id, w.max_draft_len, out=out)
+    torch.cuda.synchronize()
+    print(json.dumps({"stage1_only": w.name, "frames": int(cb.logits.shape[0]), "V_ctc": w.V_ctc,
+                      "dtype": w.dtype, "calls": 3}))
+
+
 def main():
     args = parse_args()
     if args.sweep:
         run_sweep(args)
+        return
+    if args.ncu_stage1:
+        run_stage1_only(args)
         return
     if args.impl == "reference":
         run_reference(args)
