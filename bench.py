@@ -457,7 +457,43 @@ def time_next_rows(sets, device, peak):
              "same_decisions_as_full": bool(same),
              "note": "separate mode, not part of `value`: rows after an utterance's first reject "
                      "are not read (Section 2.3 needs only the first reject)"}
-    return {"early_exit_step": early, "threshold_sweep": {"pairs": len(pairs), "us_per_call": round(t_sw, 2)},
+    # one rank's share of a vocabulary-parallel head: a quarter of the columns, then the
+    # combination of four ranks' statistics (this GPU's own four slices stand in for them; the
+    # all-gather between ranks, 12 bytes per row, needs more than one GPU and is not timed)
+    vp = None
+    if w.V_llm % 4 == 0:
+        vq = w.V_llm // 4
+        vsh = []
+        for s in sets:
+            ws = torch.empty((max(256, ssd.ssd_verify_workspace_bytes(s["B"], s["M"], vq, code)),),
+                             dtype=torch.uint8, device=device)
+            st = torch.zeros((4, s["M"], 3), dtype=torch.float32, device=device)
+            for r in range(4):
+                ssd.ssd_verify_shard(s["vb"].logits[:, r * vq:(r + 1) * vq], r * vq, s["tok_off"],
+                                     s["ids"], skip=s["gate"]["gate_accept"], stats=st[r],
+                                     workspace=ws)
+            o = ssd.alloc_verify_outputs(s["M"], s["B"], device, 0)
+            ssd.ssd_verify_combine(st, w.V_llm, s["tok_off"], s["ids"], w.tau_slm,
+                                   skip=s["gate"]["gate_accept"], out=o)
+            vsh.append((ws, st, o))
+        torch.cuda.synchronize()
+        same_vp = all(torch.equal(vsh[i][2]["accepted_len"], sets[i]["s2"]["accepted_len"])
+                      for i in range(n_sets))
+        t_sh = timed(lambda i: ssd.ssd_verify_shard(
+            sets[i]["vb"].logits[:, vq:2 * vq], vq, sets[i]["tok_off"], sets[i]["ids"],
+            skip=sets[i]["gate"]["gate_accept"], stats=vsh[i][1][1], workspace=vsh[i][0]), n_ee)
+        t_cb = timed(lambda i: ssd.ssd_verify_combine(
+            vsh[i][1], w.V_llm, sets[i]["tok_off"], sets[i]["ids"], w.tau_slm,
+            skip=sets[i]["gate"]["gate_accept"], out=vsh[i][2]))
+        sh_bytes = rows_full / n_sets * vq * (2 if w.dtype == "bf16" else 4)
+        vp = {"ranks": 4, "shard_us": round(t_sh, 2), "combine_us": round(t_cb, 2),
+              "shard_gbs": round(sh_bytes / (t_sh * 1e-6) / 1e9, 1),
+              "same_decisions_as_full": bool(same_vp),
+              "note": "ssd_verify_shard on columns [V/4, V/2) (host-paced call: streaming kernel "
+                      "plus its closing kernel) and ssd_verify_combine over four slices' "
+                      "statistics; the all-gather between ranks is not part of it"}
+    return {"early_exit_step": early, "vocab_parallel_verify": vp,
+            "threshold_sweep": {"pairs": len(pairs), "us_per_call": round(t_sw, 2)},
             "assemble": {"us_per_call": round(t_asm, 2),
                          "ar_count": int(prep[0][1]["ar_count"].cpu()[0])},
             "greedy_step": {"rows": R, "V": w.V_llm, "us_per_call": round(t_gr, 2),

@@ -317,6 +317,44 @@ int32_t ssd_verify_static(const void *logits, ssd_dtype dtype, int32_t V, int64_
                           void *stream, const ssd_launch_opts *opts);
 
 /*
+ * Stage 2 over a vocabulary-parallel LLM head.  Eq. 5 of the paper needs, per draft position,
+ * the softmax over the whole LLM vocabulary; when the head's columns are split over R ranks
+ * (tensor parallelism), each rank holds logits[:, col0 : col0 + V_local] and the log-sum-exp
+ * needs one exchange.  (The paper runs on one GPU and has no such step; the arithmetic is Eq. 5's.)
+ *
+ * ssd_verify_shard, on every rank: for each row i of a verified utterance
+ *   shard_stats[3*i + 0] = max over the local columns of x_iv
+ *   shard_stats[3*i + 1] = sum over the local columns of exp(x_iv - that maximum)
+ *   shard_stats[3*i + 2] = x[i, draft_ids[i] - col0] if col0 <= draft_ids[i] < col0 + V_local,
+ *                          else -inf            (draft_ids are ids in the whole vocabulary)
+ * Rows of skipped (or malformed) utterances are not read and their triples are left untouched.
+ * logits [M, ld] dtype (this rank's columns), shard_stats [M, 3] f32, workspace as for
+ * ssd_verify with V = V_local (ssd_verify_workspace_bytes(B, M, V_local, dtype, opts)).
+ *
+ * The exchange is the caller's: an all-gather of the R ranks' shard_stats (12 bytes per row)
+ * into stats_all [R, M, 3], rank-major, with whatever collective library it uses.
+ *
+ * ssd_verify_combine, on any rank that wants the decisions: per row
+ *   row_lse[i]    = log sum_r shard sums re-based to the global maximum          (nullable)
+ *   token_logp[i] = (the draft token's logit, from the rank that owns it) - row_lse[i]
+ * then acceptance, accepted_len, all_accepted and utt_status exactly as ssd_verify (a draft id
+ * outside [0, V_total) is a rejected position and sets SSD_UTT_BAD_DRAFT_ID).
+ * R = 1 with col0 = 0 reproduces ssd_verify.
+ * Errors: as ssd_verify; SSD_ERR_ARG also for col0 < 0, R < 1 or V_total < 1.
+ */
+int32_t ssd_verify_shard(const void *logits, ssd_dtype dtype, int32_t V_local, int64_t ld,
+                         int64_t col0, const int64_t *tok_off, const int32_t *draft_ids,
+                         int32_t B, int64_t M, const uint8_t *skip, float *shard_stats,
+                         void *workspace, size_t workspace_bytes, void *stream,
+                         const ssd_launch_opts *opts);
+int32_t ssd_verify_combine(const float *stats_all, int32_t R, int64_t V_total,
+                           const int64_t *tok_off, const int32_t *draft_ids, int32_t B, int64_t M,
+                           float tau_slm, const uint8_t *skip,
+                           float *token_logp, float *row_lse,
+                           int32_t *accepted_len, uint8_t *all_accepted, uint32_t *utt_status,
+                           void *stream);
+
+/*
  * Read-span hooks.  The paper has no counterpart: these are test hooks of this library, host
  * only (no GPU, no stream; base_addr is an integer that is never dereferenced).
  *

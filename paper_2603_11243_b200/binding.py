@@ -76,6 +76,12 @@ def lib():
             f.restype = i32
         L.ssd_ctc_draft_read_span.argtypes = [C.c_uint64, C.c_int, i32, i64, i64, vp, vp]
         L.ssd_verify_read_span.argtypes = [C.c_uint64, C.c_int, i32, i64, i64, i32, vp, vp]
+        L.ssd_verify_shard.restype = i32
+        L.ssd_verify_shard.argtypes = [vp, C.c_int, i32, i64, i64, vp, vp, i32, i64, vp, vp, vp,
+                                       C.c_size_t, vp, vp]
+        L.ssd_verify_combine.restype = i32
+        L.ssd_verify_combine.argtypes = [vp, i32, i64, vp, vp, i32, i64, C.c_float, vp, vp, vp, vp,
+                                         vp, vp, vp]
         L.ssd_threshold_sweep.restype = i32
         L.ssd_threshold_sweep.argtypes = [vp, vp, vp, i32, i64, vp, vp, i32, vp, vp, vp, vp, vp]
         L.ssd_assemble.restype = i32
@@ -276,6 +282,59 @@ def ssd_verify_static(logits: torch.Tensor, tok_off: torch.Tensor, draft_ids: to
         _dev(out["utt_status"], "utt_status"), _stream(), _opts(opts))
     if rc != OK:
         raise SsdError(rc, "ssd_verify_static")
+    return out
+
+
+def ssd_verify_shard(logits: torch.Tensor, col0: int, tok_off: torch.Tensor,
+                     draft_ids: torch.Tensor, skip: Optional[torch.Tensor] = None,
+                     V_local: Optional[int] = None, stats: Optional[torch.Tensor] = None,
+                     workspace: Optional[torch.Tensor] = None,
+                     opts: Optional[LaunchOpts] = None) -> torch.Tensor:
+    """Stage 2 over a vocabulary-parallel LLM head, this rank's part: `logits` holds columns
+    [col0, col0 + V_local) of the whole vocabulary; returns [M, 3] (max, sum, draft logit)."""
+    M, ld = _rows_ld(logits)
+    V_local = logits.shape[1] if V_local is None else V_local
+    B = tok_off.shape[0] - 1
+    if tok_off.dtype != torch.int64 or draft_ids.dtype != torch.int32:
+        raise TypeError("tok_off must be int64 and draft_ids int32")
+    if skip is not None and skip.dtype != torch.uint8:
+        raise TypeError("skip must be uint8")
+    if stats is None:
+        stats = torch.zeros((M, 3), dtype=torch.float32, device=logits.device)
+    if workspace is None:
+        need = ssd_verify_workspace_bytes(B, M, V_local, _dtype_code(logits), opts)
+        workspace = torch.empty((max(need, 256),), dtype=torch.uint8, device=logits.device)
+    rc = lib().ssd_verify_shard(
+        _dev(logits, "logits"), _dtype_code(logits), V_local, ld, col0, _dev(tok_off, "tok_off"),
+        _dev(draft_ids, "draft_ids"), B, M, _dev(skip, "skip"), _dev(stats, "shard_stats"),
+        _dev(workspace, "workspace"), workspace.numel(), _stream(), _opts(opts))
+    if rc != OK:
+        raise SsdError(rc, "ssd_verify_shard")
+    return stats
+
+
+def ssd_verify_combine(stats_all: torch.Tensor, V_total: int, tok_off: torch.Tensor,
+                       draft_ids: torch.Tensor, tau_slm: float,
+                       skip: Optional[torch.Tensor] = None, out=None) -> Dict[str, torch.Tensor]:
+    """After the all-gather of every rank's ssd_verify_shard result into stats_all [R, M, 3]:
+    log-likelihoods (Eq. 5) and the accepted prefix, as ssd_verify returns them."""
+    if stats_all.dim() != 3 or stats_all.shape[2] != 3 or not stats_all.is_contiguous() \
+            or stats_all.dtype != torch.float32:
+        raise ValueError("stats_all must be a contiguous float32 tensor [R, M, 3]")
+    R, M = stats_all.shape[0], stats_all.shape[1]
+    B = tok_off.shape[0] - 1
+    if tok_off.dtype != torch.int64 or draft_ids.dtype != torch.int32:
+        raise TypeError("tok_off must be int64 and draft_ids int32")
+    if out is None:
+        out = alloc_verify_outputs(M, B, stats_all.device, 0)
+    rc = lib().ssd_verify_combine(
+        _dev(stats_all, "stats_all"), R, V_total, _dev(tok_off, "tok_off"),
+        _dev(draft_ids, "draft_ids"), B, M, C.c_float(tau_slm), _dev(skip, "skip"),
+        _dev(out["token_logp"], "token_logp"), _dev(out.get("row_lse"), "row_lse"),
+        _dev(out["accepted_len"], "accepted_len"), _dev(out["all_accepted"], "all_accepted"),
+        _dev(out["utt_status"], "utt_status"), _stream())
+    if rc != OK:
+        raise SsdError(rc, "ssd_verify_combine")
     return out
 
 

@@ -110,6 +110,42 @@ int32_t ssd_verify(const void *logits, ssd_dtype dtype, int32_t V, int64_t ld,
                          token_logp, row_lse, accepted_len, all_accepted, utt_status, plan, L);
 }
 
+int32_t ssd_verify_shard(const void *logits, ssd_dtype dtype, int32_t V_local, int64_t ld,
+                         int64_t col0, const int64_t *tok_off, const int32_t *draft_ids,
+                         int32_t B, int64_t M, const uint8_t *skip, float *shard_stats,
+                         void *workspace, size_t workspace_bytes, void *stream,
+                         const ssd_launch_opts *opts) {
+    if (dtype != SSD_F32 && dtype != SSD_BF16) return SSD_ERR_DTYPE;
+    if (B < 0 || M < 0 || V_local < 1 || ld < V_local || col0 < 0) return SSD_ERR_ARG;
+    if (!tok_off) return SSD_ERR_NULL;
+    if (M > 0 && (!logits || !draft_ids || !shard_stats)) return SSD_ERR_NULL;
+    const int es = dtype == SSD_F32 ? 4 : 2;
+    if (reinterpret_cast<uintptr_t>(logits) % es) return SSD_ERR_ALIGN;
+    VerifyPlan plan;
+    int rc = plan_verify(B, M, V_local, dtype, opts, &plan);
+    if (rc != SSD_OK) return rc;
+    if (B > 0 && (!workspace || workspace_bytes < plan.workspace_bytes ||
+                  reinterpret_cast<uintptr_t>(workspace) % 256))
+        return SSD_ERR_WORKSPACE;
+    Launch L{static_cast<cudaStream_t>(stream), opts};
+    return launch_verify_shard(logits, dtype, V_local, ld, M, col0, tok_off, draft_ids, B, skip,
+                               workspace, shard_stats, plan, L);
+}
+
+int32_t ssd_verify_combine(const float *stats_all, int32_t R, int64_t V_total,
+                           const int64_t *tok_off, const int32_t *draft_ids, int32_t B, int64_t M,
+                           float tau_slm, const uint8_t *skip,
+                           float *token_logp, float *row_lse,
+                           int32_t *accepted_len, uint8_t *all_accepted, uint32_t *utt_status,
+                           void *stream) {
+    if (B < 0 || M < 0 || R < 1 || V_total < 1) return SSD_ERR_ARG;
+    if (!tok_off || (B > 0 && (!accepted_len || !all_accepted || !utt_status))) return SSD_ERR_NULL;
+    if (M > 0 && (!stats_all || !draft_ids || !token_logp)) return SSD_ERR_NULL;
+    return launch_verify_combine(stats_all, R, V_total, tok_off, draft_ids, B, M, tau_slm, skip,
+                                 token_logp, row_lse, accepted_len, all_accepted, utt_status,
+                                 static_cast<cudaStream_t>(stream));
+}
+
 int32_t ssd_threshold_sweep(const float *utt_max_entropy, const float *token_logp,
                             const int64_t *tok_off, int32_t B, int64_t M,
                             const float *tau_ctc, const float *tau_slm, int32_t P,

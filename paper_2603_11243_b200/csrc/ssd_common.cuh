@@ -358,6 +358,15 @@ struct VerifyPlan {
 };
 int plan_verify(int B, int64_t M, int V, ssd_dtype dtype, const ssd_launch_opts *opts,
                 VerifyPlan *plan);
+int launch_verify_shard(const void *logits, ssd_dtype dtype, int V_local, int64_t ld, int64_t M,
+                        int64_t col0, const int64_t *tok_off, const int32_t *draft_ids, int B,
+                        const uint8_t *skip, void *workspace, float *shard_stats,
+                        const VerifyPlan &plan, const Launch &L);
+int launch_verify_combine(const float *stats_all, int R, int64_t V_total, const int64_t *tok_off,
+                          const int32_t *draft_ids, int B, int64_t M, float tau_slm,
+                          const uint8_t *skip, float *token_logp, float *row_lse,
+                          int32_t *accepted_len, uint8_t *all_accepted, uint32_t *utt_status,
+                          cudaStream_t stream);
 int launch_verify(const void *logits, ssd_dtype dtype, int V, int64_t ld, int64_t M,
                   const int64_t *tok_off, const int32_t *draft_ids, int B, float tau_slm,
                   const uint8_t *skip, void *workspace, float *token_logp, float *row_lse,

@@ -344,6 +344,137 @@ __global__ void __launch_bounds__(kFinishThreads) verify_finish_kernel(
     }
 }
 
+// Merge of a row's P (reference, sum) pairs into (maximum, sum relative to it).
+__device__ __forceinline__ float2 merge_partials(const float2 *pp, int P) {
+    float Mx = kNegInit, S = 0.f;
+    if ((P & 1) == 0 && P <= 16) {
+        const float4 *p4 = reinterpret_cast<const float4 *>(pp);
+        float4 v[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+            v[q] = q < P / 2 ? p4[q] : make_float4(kNegInit, 0.f, kNegInit, 0.f);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) Mx = fmaxf(Mx, fmaxf(v[q].x, v[q].z));
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+            S += v[q].y * ex2((v[q].x - Mx) * kLog2e) + v[q].w * ex2((v[q].z - Mx) * kLog2e);
+    } else {
+        for (int q = 0; q < P; ++q) Mx = fmaxf(Mx, pp[q].x);
+        for (int q = 0; q < P; ++q) {
+            const float2 v = pp[q];
+            S += v.y * ex2((v.x - Mx) * kLog2e);
+        }
+    }
+    return make_float2(Mx, S);
+}
+
+constexpr uint32_t kStatsInternal = 0x7fc0dead;   // in place of a row's maximum: a wait ran out
+
+// Vocabulary-parallel verification, per rank: for every row of a verified utterance the
+// triple (maximum of the local columns, sum of exponentials relative to it, logit of the draft
+// token if its column is local, else -inf).  Rows of skipped or malformed utterances are left
+// untouched; the combining kernel does not read them.
+template <typename T>
+__global__ void __launch_bounds__(kFinishThreads) shard_finish_kernel(
+    const char *__restrict__ logits, int V_local, int64_t ld, int64_t M, int64_t col0,
+    const int64_t *__restrict__ tok_off, const int32_t *__restrict__ draft_ids, int B,
+    const uint8_t *__restrict__ skip, const float2 *__restrict__ partials, int P,
+    float *__restrict__ stats, const unsigned long long *err_word, unsigned long long epoch) {
+    constexpr int ES = Elem<T>::kBytes;
+    pdl_enter();
+    const int b = blockIdx.x, tid = threadIdx.x;
+    const int64_t i0 = tok_off[b], i1 = tok_off[b + 1];
+    const unsigned long long err = *err_word;
+    const bool skipped = skip != nullptr && skip[b] != 0;
+    if (i0 < 0 || i1 < i0 || i1 > M || skipped) return;
+    const bool internal = err == epoch;
+    for (int64_t r = i0 + tid; r < i1; r += blockDim.x) {
+        const int64_t local = (int64_t)draft_ids[r] - col0;
+        const bool owned = local >= 0 && local < V_local;
+        float x = -INFINITY;
+        if (owned) x = Elem<T>::load(logits + (r * ld + local) * ES);
+        const float2 ms = merge_partials(partials + r * P, P);
+        stats[3 * r + 0] = internal ? __uint_as_float(kStatsInternal) : ms.x;
+        stats[3 * r + 1] = ms.y;
+        stats[3 * r + 2] = x;
+    }
+}
+
+// Vocabulary-parallel verification, after the exchange: stats_all holds R ranks' triples,
+// [R, M, 3].  Per row the global maximum, the sum re-based to it, the draft token's logit (the
+// one shard that owns the column has it), then Eq. 5 and the first reject exactly as in
+// verify_finish_kernel.
+__global__ void __launch_bounds__(kFinishThreads) combine_kernel(
+    const float *__restrict__ stats_all, int R, int64_t V_total, int64_t M,
+    const int64_t *__restrict__ tok_off, const int32_t *__restrict__ draft_ids, int B,
+    float log_tau, int reject_none, const uint8_t *__restrict__ skip,
+    float *__restrict__ token_logp, float *__restrict__ row_lse,
+    int32_t *__restrict__ accepted_len, uint8_t *__restrict__ all_accepted,
+    uint32_t *__restrict__ utt_status) {
+    __shared__ int first_reject;
+    __shared__ unsigned flags;
+    pdl_enter();
+    const int b = blockIdx.x, tid = threadIdx.x;
+    const int64_t i0 = tok_off[b], i1 = tok_off[b + 1];
+    const bool skipped = skip != nullptr && skip[b] != 0;
+    if (i0 < 0 || i1 < i0 || i1 > M) {
+        if (tid == 0) { accepted_len[b] = 0; all_accepted[b] = 0; utt_status[b] = SSD_UTT_BAD_OFFSETS; }
+        return;
+    }
+    const int64_t K64 = i1 - i0;
+    const int K = K64 > 0x7fffffff ? 0x7fffffff : (int)K64;
+    if (skipped) {
+        if (tid == 0) { accepted_len[b] = K; all_accepted[b] = 1; utt_status[b] = 0; }
+        return;
+    }
+    if (tid == 0) { first_reject = K; flags = 0; }
+    __syncthreads();
+    unsigned myflags = 0;
+    int myfirst = K;
+    for (int i = tid; i < K; i += blockDim.x) {
+        const int64_t r = i0 + i;
+        const int id = draft_ids[r];
+        const bool id_ok = id >= 0 && (int64_t)id < V_total;
+        float Mx = kNegInit, x = -INFINITY;
+        for (int q = 0; q < R; ++q) {
+            const float *t = stats_all + ((int64_t)q * M + r) * 3;
+            const float m = t[0];
+            if (__float_as_uint(m) == kStatsInternal) myflags |= SSD_UTT_INTERNAL;
+            Mx = fmaxf(Mx, m);
+            x = fmaxf(x, t[2]);
+        }
+        float S = 0.f;
+        for (int q = 0; q < R; ++q) {
+            const float *t = stats_all + ((int64_t)q * M + r) * 3;
+            S += t[1] * ex2((t[0] - Mx) * kLog2e);
+        }
+        const float lnS = logf(S);
+        const float lse = Mx + lnS;
+        if (!(fabsf(lse) < INFINITY)) myflags |= SSD_UTT_NONFINITE;
+        float logp;
+        bool reject;
+        if (!id_ok) {
+            myflags |= SSD_UTT_BAD_DRAFT_ID;
+            logp = -INFINITY;
+            reject = true;
+        } else {
+            logp = (x - Mx) - lnS;
+            reject = reject_none ? false : !(logp > log_tau);
+        }
+        token_logp[r] = logp;
+        if (row_lse) row_lse[r] = lse;
+        if (reject && i < myfirst) myfirst = i;
+    }
+    if (myfirst < K) atomicMin(&first_reject, myfirst);
+    if (myflags) atomicOr(&flags, myflags);
+    __syncthreads();
+    if (tid == 0) {
+        accepted_len[b] = first_reject;
+        all_accepted[b] = first_reject == K ? 1 : 0;
+        utt_status[b] = flags;
+    }
+}
+
 // Greedy step: merges the partials of a row, one warp per row.  A partial is
 // (reference, sum, largest logit, index of its first occurrence).
 constexpr int kGreedyWarps = 8;
@@ -450,65 +581,121 @@ int plan_verify(int B, int64_t M, int V, ssd_dtype dtype, const ssd_launch_opts 
     return SSD_OK;
 }
 
+// Launches the streaming kernel that leaves plan.partials (reference, sum) pairs per row in the
+// workspace (nothing for rows of skipped utterances).
+static int launch_verify_rows(const void *logits, ssd_dtype dtype, int V, int64_t ld, int64_t M,
+                              const int64_t *tok_off, int B, const uint8_t *skip, void *workspace,
+                              unsigned long long epoch, const VerifyPlan &plan, const Launch &L) {
+    if (M == 0) return SSD_OK;
+    const ssd_launch_opts *o = L.opts;
+    cudaError_t e;
+    VerifyParams p{};
+    p.logits = static_cast<const char *>(logits);
+    p.V = V; p.ld = ld; p.M = M; p.split = plan.split; p.num_items = M * plan.split;
+    p.tok_off = tok_off; p.B = B; p.skip = skip;
+    p.partials = reinterpret_cast<float2 *>(static_cast<char *>(workspace) + 256);
+    p.partials_per_row = plan.partials;
+    p.warps = plan.warps; p.stages = plan.stages; p.stage_bytes = plan.stage_bytes;
+    p.err_word = static_cast<unsigned long long *>(workspace); p.epoch = epoch;
+    int64_t ctas = p.num_items < plan.ctas ? p.num_items : plan.ctas;
+    if (o && o->ev_begin) {
+        e = cudaEventRecord(static_cast<cudaEvent_t>(o->ev_begin), L.stream);
+        if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
+    }
+    if (plan.kernel == 2) {
+        void (*kern)(const VerifyParams) = verify_rows_tma<float, 0, false>;
+        if (dtype == SSD_BF16)
+            kern = plan.fma_exp == 1 ? verify_rows_tma<bf16_t, 1, false>
+                 : plan.fma_exp == 2 ? verify_rows_tma<bf16_t, 2, false>
+                 : plan.fma_exp == 3 ? verify_rows_tma<bf16_t, 3, false>
+                                     : verify_rows_tma<bf16_t, 0, false>;
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)plan.smem_bytes);
+        if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
+        e = launch_pdl(kern, (unsigned)ctas, (unsigned)((plan.warps + 1) * 32), plan.smem_bytes,
+                       L.stream, p);
+        if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
+    } else {
+        ctas = p.num_items < 8ll * plan.ctas ? p.num_items : 8ll * plan.ctas;
+        e = launch_pdl(dtype == SSD_F32 ? verify_rows_plain<float> : verify_rows_plain<bf16_t>,
+                       (unsigned)ctas, 256u, 0, L.stream, p);
+        if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
+    }
+    e = cudaGetLastError();
+    if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
+    if (o && o->ev_end) {
+        e = cudaEventRecord(static_cast<cudaEvent_t>(o->ev_end), L.stream);
+        if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
+    }
+    return SSD_OK;
+}
+
 int launch_verify(const void *logits, ssd_dtype dtype, int V, int64_t ld, int64_t M,
                   const int64_t *tok_off, const int32_t *draft_ids, int B, float tau_slm,
                   const uint8_t *skip, void *workspace, float *token_logp, float *row_lse,
                   int32_t *accepted_len, uint8_t *all_accepted, uint32_t *utt_status,
                   const VerifyPlan &plan, const Launch &L) {
     if (B == 0) return SSD_OK;
-    const ssd_launch_opts *o = L.opts;
     unsigned long long *err_word = static_cast<unsigned long long *>(workspace);
     float2 *partials = reinterpret_cast<float2 *>(static_cast<char *>(workspace) + 256);
     const unsigned long long epoch = next_epoch();
-    cudaError_t e;
-    if (M > 0) {
-        VerifyParams p{};
-        p.logits = static_cast<const char *>(logits);
-        p.V = V; p.ld = ld; p.M = M; p.split = plan.split; p.num_items = M * plan.split;
-        p.tok_off = tok_off; p.B = B; p.skip = skip;
-        p.partials = partials; p.partials_per_row = plan.partials;
-        p.warps = plan.warps; p.stages = plan.stages; p.stage_bytes = plan.stage_bytes;
-        p.err_word = err_word; p.epoch = epoch;
-        int64_t ctas = p.num_items < plan.ctas ? p.num_items : plan.ctas;
-        if (o && o->ev_begin) {
-            e = cudaEventRecord(static_cast<cudaEvent_t>(o->ev_begin), L.stream);
-            if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
-        }
-        if (plan.kernel == 2) {
-            void (*kern)(const VerifyParams) = verify_rows_tma<float, 0, false>;
-            if (dtype == SSD_BF16)
-                kern = plan.fma_exp == 1 ? verify_rows_tma<bf16_t, 1, false>
-                     : plan.fma_exp == 2 ? verify_rows_tma<bf16_t, 2, false>
-                     : plan.fma_exp == 3 ? verify_rows_tma<bf16_t, 3, false>
-                                         : verify_rows_tma<bf16_t, 0, false>;
-            e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)plan.smem_bytes);
-            if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
-            e = launch_pdl(kern, (unsigned)ctas, (unsigned)((plan.warps + 1) * 32), plan.smem_bytes,
-                           L.stream, p);
-            if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
-        } else {
-            ctas = p.num_items < 8ll * plan.ctas ? p.num_items : 8ll * plan.ctas;
-            e = launch_pdl(dtype == SSD_F32 ? verify_rows_plain<float> : verify_rows_plain<bf16_t>,
-                           (unsigned)ctas, 256u, 0, L.stream, p);
-            if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
-        }
-        e = cudaGetLastError();
-        if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
-        if (o && o->ev_end) {
-            e = cudaEventRecord(static_cast<cudaEvent_t>(o->ev_end), L.stream);
-            if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
-        }
-    }
+    const int rc = launch_verify_rows(logits, dtype, V, ld, M, tok_off, B, skip, workspace, epoch,
+                                      plan, L);
+    if (rc != SSD_OK) return rc;
     const double tau = (double)tau_slm;
     const int reject_none = !(tau > 0.0);
     const float log_tau = reject_none ? -INFINITY : (float)log(tau);
-    e = launch_pdl(dtype == SSD_F32 ? verify_finish_kernel<float> : verify_finish_kernel<bf16_t>,
-                   (unsigned)B, (unsigned)kFinishThreads, 0, L.stream,
-                   static_cast<const char *>(logits), V, ld, M, tok_off, draft_ids, B, log_tau,
-                   reject_none, skip, static_cast<const float2 *>(partials), plan.partials,
-                   token_logp, row_lse, accepted_len, all_accepted, utt_status,
-                   static_cast<const unsigned long long *>(err_word), epoch);
+    cudaError_t e = launch_pdl(
+        dtype == SSD_F32 ? verify_finish_kernel<float> : verify_finish_kernel<bf16_t>,
+        (unsigned)B, (unsigned)kFinishThreads, 0, L.stream,
+        static_cast<const char *>(logits), V, ld, M, tok_off, draft_ids, B, log_tau,
+        reject_none, skip, static_cast<const float2 *>(partials), plan.partials,
+        token_logp, row_lse, accepted_len, all_accepted, utt_status,
+        static_cast<const unsigned long long *>(err_word), epoch);
+    if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
+    e = cudaGetLastError();
+    if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
+    return SSD_OK;
+}
+
+// Vocabulary-parallel verification, this rank's part: the same streaming kernel over the local
+// columns, then one (maximum, sum, draft logit) triple per row.
+int launch_verify_shard(const void *logits, ssd_dtype dtype, int V_local, int64_t ld, int64_t M,
+                        int64_t col0, const int64_t *tok_off, const int32_t *draft_ids, int B,
+                        const uint8_t *skip, void *workspace, float *shard_stats,
+                        const VerifyPlan &plan, const Launch &L) {
+    if (B == 0) return SSD_OK;
+    unsigned long long *err_word = static_cast<unsigned long long *>(workspace);
+    float2 *partials = reinterpret_cast<float2 *>(static_cast<char *>(workspace) + 256);
+    const unsigned long long epoch = next_epoch();
+    const int rc = launch_verify_rows(logits, dtype, V_local, ld, M, tok_off, B, skip, workspace,
+                                      epoch, plan, L);
+    if (rc != SSD_OK) return rc;
+    cudaError_t e = launch_pdl(
+        dtype == SSD_F32 ? shard_finish_kernel<float> : shard_finish_kernel<bf16_t>,
+        (unsigned)B, (unsigned)kFinishThreads, 0, L.stream,
+        static_cast<const char *>(logits), V_local, ld, M, col0, tok_off, draft_ids, B, skip,
+        static_cast<const float2 *>(partials), plan.partials, shard_stats,
+        static_cast<const unsigned long long *>(err_word), epoch);
+    if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
+    e = cudaGetLastError();
+    if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
+    return SSD_OK;
+}
+
+int launch_verify_combine(const float *stats_all, int R, int64_t V_total, const int64_t *tok_off,
+                          const int32_t *draft_ids, int B, int64_t M, float tau_slm,
+                          const uint8_t *skip, float *token_logp, float *row_lse,
+                          int32_t *accepted_len, uint8_t *all_accepted, uint32_t *utt_status,
+                          cudaStream_t stream) {
+    if (B == 0) return SSD_OK;
+    const double tau = (double)tau_slm;
+    const int reject_none = !(tau > 0.0);
+    const float log_tau = reject_none ? -INFINITY : (float)log(tau);
+    cudaError_t e = launch_pdl(combine_kernel, (unsigned)B, (unsigned)kFinishThreads, 0, stream,
+                               stats_all, R, V_total, M, tok_off, draft_ids, B, log_tau,
+                               reject_none, skip, token_logp, row_lse, accepted_len, all_accepted,
+                               utt_status);
     if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
     e = cudaGetLastError();
     if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }

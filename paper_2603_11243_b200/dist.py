@@ -67,3 +67,24 @@ def reduce_max_sum(local_max: float, local_sum: float, device) -> Tuple[float, f
     dist.all_reduce(m, op=dist.ReduceOp.MAX)
     dist.all_reduce(s, op=dist.ReduceOp.SUM)
     return float(m.item()), float(s.item())
+
+
+def all_gather_rows(local: torch.Tensor) -> torch.Tensor:
+    """[R, ...] stack of every rank's `local` tensor (same shape on all ranks), rank-major: the one
+    exchange of vocabulary-parallel verification (each rank's [M, 3] partial statistics, 12 bytes
+    per row).  Without a process group the result is the local tensor with a leading 1."""
+    if not dist.is_initialized():
+        return local.unsqueeze(0).contiguous()
+    parts = [torch.empty_like(local) for _ in range(dist.get_world_size())]
+    dist.all_gather(parts, local.contiguous())
+    return torch.stack(parts).contiguous()
+
+
+def vocab_shard(V_total: int, rank: int, world: int, multiple: int = 8) -> Tuple[int, int]:
+    """(col0, V_local) of rank's slice when V_total columns are split as evenly as possible in
+    units of `multiple` columns (the last rank takes the remainder)."""
+    units = (V_total + multiple - 1) // multiple
+    lo = (units * rank // world) * multiple
+    hi = V_total if rank == world - 1 else (units * (rank + 1) // world) * multiple
+    return lo, max(0, min(hi, V_total) - lo)
+

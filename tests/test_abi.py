@@ -173,3 +173,26 @@ def test_early_exit_rejects_bad_arguments_on_the_host(lib):
         assert ee(*bad) == code, (i, v)
     full = ssd.ssd_verify_workspace_bytes(64, 20000, 49152, ssd.BF16)
     assert ssd.ssd_verify_early_exit_workspace_bytes(64, 20000, 49152, ssd.BF16) >= full
+
+
+def test_vocab_parallel_calls_reject_bad_arguments_on_the_host(lib):
+    p = lambda n: C.c_void_p(n)
+    f32 = C.c_float(0.1)
+    sh = lambda logits, dtype, V, ld, col0, off, ids, B, M, stats, ws, wsb: lib.ssd_verify_shard(
+        logits, dtype, V, ld, col0, off, ids, B, M, None, stats, ws, wsb, None, None)
+    assert sh(p(8), 9, 10, 10, 0, p(8), p(8), 1, 4, p(8), p(256), 1 << 20) == ssd.ERR_DTYPE
+    assert sh(p(8), 1, 10, 9, 0, p(8), p(8), 1, 4, p(8), p(256), 1 << 20) == ssd.ERR_ARG     # ld < V
+    assert sh(p(8), 1, 10, 10, -1, p(8), p(8), 1, 4, p(8), p(256), 1 << 20) == ssd.ERR_ARG   # col0 < 0
+    assert sh(p(8), 1, 10, 10, 0, None, p(8), 1, 4, p(8), p(256), 1 << 20) == ssd.ERR_NULL
+    assert sh(p(8), 1, 10, 10, 0, p(8), p(8), 1, 4, None, p(256), 1 << 20) == ssd.ERR_NULL
+    assert sh(p(9), 1, 10, 10, 0, p(8), p(8), 1, 4, p(8), p(256), 1 << 20) == ssd.ERR_ALIGN
+    assert sh(p(8), 1, 10, 10, 0, p(8), p(8), 1, 4, p(8), p(256), 16) == ssd.ERR_WORKSPACE
+    assert sh(p(8), 1, 10, 10, 0, p(8), p(8), 0, 0, p(8), None, 0) == ssd.OK                # nothing to do
+    cb = lambda stats, R, V, off, ids, B, M, lp, al, aa, st: lib.ssd_verify_combine(
+        stats, R, V, off, ids, B, M, f32, None, lp, None, al, aa, st, None)
+    assert cb(p(8), 0, 10, p(8), p(8), 1, 4, p(8), p(8), p(8), p(8)) == ssd.ERR_ARG          # R < 1
+    assert cb(p(8), 2, 0, p(8), p(8), 1, 4, p(8), p(8), p(8), p(8)) == ssd.ERR_ARG           # V < 1
+    assert cb(None, 2, 10, p(8), p(8), 1, 4, p(8), p(8), p(8), p(8)) == ssd.ERR_NULL
+    assert cb(p(8), 2, 10, p(8), p(8), 1, 4, p(8), None, p(8), p(8)) == ssd.ERR_NULL
+    assert cb(p(8), 2, 10, p(8), p(8), 0, 0, p(8), p(8), p(8), p(8)) == ssd.OK
+

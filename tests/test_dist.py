@@ -24,6 +24,24 @@ def test_partition_by_bytes_is_contiguous_and_balanced():
     assert D.partition_by_bytes([], 3) == [(0, 0)] * 3
 
 
+def test_vocab_shards_tile_the_vocabulary():
+    for V in (1, 7, 8, 9, 1001, 49152, 152064):
+        for world in (1, 2, 3, 8):
+            spans = [D.vocab_shard(V, r, world) for r in range(world)]
+            at = 0
+            for col0, n in spans:
+                assert n >= 0 and (n == 0 or col0 == at)
+                at += n
+            assert at == V
+            assert all(col0 % 8 == 0 for col0, n in spans if n)
+
+
+def test_all_gather_rows_without_a_process_group():
+    import torch
+    x = torch.arange(6.0).reshape(2, 3)
+    assert torch.equal(D.all_gather_rows(x), x.unsqueeze(0))
+
+
 def test_rank_seeds_differ_and_rank0_keeps_the_workload_seed():
     assert D.rank_seed(7, 0) == 7
     assert len({D.rank_seed(7, r) for r in range(8)}) == 8
@@ -51,6 +69,15 @@ WORKER = textwrap.dedent("""
     spans = [None, None]
     torch.distributed.all_gather_object(spans, (lo, hi))
     assert spans[0][1] == spans[1][0] and spans[0][0] == 0 and spans[1][1] == len(costs)
+    # the exchange of vocabulary-parallel verification: every rank's [M, 3] statistics, rank-major
+    V_total = 1001
+    col0, v_local = D.vocab_shard(V_total, rank, world)
+    mine = torch.full((5, 3), float(rank)) + torch.arange(15.0).reshape(5, 3) / 100
+    mine[:, 2] = col0
+    allr = D.all_gather_rows(mine)
+    assert tuple(allr.shape) == (2, 5, 3) and allr.is_contiguous()
+    assert torch.equal(allr[rank], mine) and allr[1 - rank][0, 0] == float(1 - rank)
+    assert allr[0][0, 2] == 0 and allr[1][0, 2] == D.vocab_shard(V_total, 1, world)[0]
     D.finalize()
     sys.stdout.write("rank%%d-ok\\n" %% rank)
 """)
