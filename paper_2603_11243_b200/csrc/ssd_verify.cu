@@ -534,9 +534,12 @@ int plan_verify(int B, int64_t M, int V, ssd_dtype dtype, const ssd_launch_opts 
     int split = 1;
     if (o && o->split > 0) {
         split = o->split;
-    } else if (M > 0 && M < 8ll * pl.ctas) {
-        const int64_t want = (8ll * pl.ctas + M - 1) / M;
-        const int64_t most = row_bytes / 16384 > 1 ? row_bytes / 16384 : 1;  // spans >= 16 KB
+    } else if (M > 0 && M < 4ll * pl.ctas) {
+        // about four items per CTA, spans of 32 KB at least: every span is a stage hand-over
+        // for the consumers, so more and smaller ones lose what the better balance gains
+        // (250 rows of 98 KB: 13.9 us with 2 or 3 spans, 16.0 with 5, 16.9 with 6)
+        const int64_t want = (4ll * pl.ctas + M - 1) / M;
+        const int64_t most = row_bytes / 32768 > 1 ? row_bytes / 32768 : 1;
         split = (int)(want < most ? want : most);
     }
     if (split < 1) split = 1;
