@@ -293,8 +293,8 @@ int32_t ssd_greedy_step(const void *logits, ssd_dtype dtype, int32_t V, int64_t 
  *
  * Limit: sizes for which ssd_verify_workspace_bytes(B, M, V, dtype, opts) exceeds
  * SSD_VERIFY_STATIC_SCRATCH_BYTES are refused with SSD_ERR_TOO_LARGE before anything is
- * enqueued (with the default options the scratch is 128 bytes per logits row plus a header, so
- * about 65,000 rows fit; few rows of a wide vocabulary use more per row and still fit).
+ * enqueued (with the default options the scratch is 96 or 128 bytes per logits row plus a header,
+ * so at least 65,000 rows fit; few rows of a wide vocabulary use more per row and still fit).
  *
  * First call on a device: the function looks up the device address of the array (once per
  * device, under a lock, with the caller's current device).  Make that first call outside any
