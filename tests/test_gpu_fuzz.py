@@ -91,6 +91,44 @@ def test_stage2_random(cuda_device, seed):
     assert torch.equal(ee["all_accepted"], out["all_accepted"])
 
 
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("V", [50001, 55553, 56700, 100003, 152065])
+def test_stage2_wide_odd_rows(cuda_device, V, dtype):
+    """Rows around and above what one ring stage holds (one stage of ~100 KB per row, or two
+    or three equal parts), odd lengths, padded and misaligned.  The grid is limited to 40 CTAs
+    so that a couple of hundred rows already take the unsplit path."""
+    rng = np.random.default_rng(V)
+    B, o = 5, H.opts(ctas=40)
+    off, lens = ragged(rng, B, 90)
+    while off[-1] < 4 * 40 + 10:
+        off, lens = ragged(rng, B, 90)
+    M = int(off[-1])
+    wide, col0, ld = random_matrix(rng, M, V, dtype)
+    ids = rng.integers(0, V, size=M).astype(np.int32)
+    for r in range(M):
+        if rng.random() < 0.9:
+            wide[r, col0 + ids[r]] = 25.0
+    dev = cuda_device
+    view = wide.to(dev)[:, col0:col0 + V]
+    code = ssd.BF16 if dtype == torch.bfloat16 else ssd.F32
+    g, out = H.guarded_verify_outputs(M, B, dev, ssd.ssd_verify_workspace_bytes(B, M, V, code, o))
+    offd, idsd = torch.from_numpy(off).to(dev), torch.from_numpy(ids).to(dev)
+    ssd.ssd_verify(view, offd, idsd, 0.1, V=V, out=out, opts=o)
+    torch.cuda.synchronize()
+    g.check()
+    orc = ref.verify(H.storage_numpy(wide[:, col0:col0 + V].contiguous()), V, off, ids,
+                     float(np.float32(0.1)))
+    H.compare_stage2(out, orc, off, 0.1, require_all_margins=False)
+    ee = ssd.ssd_verify_early_exit(view, offd, idsd, 0.1, V=V, opts=o)
+    torch.cuda.synchronize()
+    assert torch.equal(ee["accepted_len"], out["accepted_len"])
+    assert bool((ee["rows_read"] >= 0).all().item())          # the position-major kernel ran
+    gr = ssd.ssd_greedy_step(view, V=V, opts=o)
+    torch.cuda.synchronize()
+    want = ref.greedy_step(H.storage_numpy(wide[:, col0:col0 + V].contiguous()), V)
+    np.testing.assert_array_equal(gr["next_token"].cpu().numpy(), want["next_token"])
+
+
 @pytest.mark.parametrize("seed", range(12))
 def test_greedy_random(cuda_device, seed):
     rng = np.random.default_rng(3000 + seed)
