@@ -19,11 +19,21 @@ def env_rank() -> Tuple[int, int, int]:
 
 
 def init(backend: str) -> Tuple[int, int, int]:
+    """Joins the process group when a launcher started this process (RANK and WORLD_SIZE in the
+    environment, a world of one included, so that a single GPU exercises the same calls); a plain
+    `python bench.py` stays without one.  With NCCL the rank's GPU is selected first and named
+    to the group, so that no collective has to guess the device."""
     rank, local_rank, world = env_rank()
-    if world > 1 and not dist.is_initialized():
+    launched = "RANK" in os.environ and "WORLD_SIZE" in os.environ
+    if launched and not dist.is_initialized():
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         os.environ.setdefault("MASTER_PORT", "29511")
-        dist.init_process_group(backend=backend, rank=rank, world_size=world)
+        if backend == "nccl":
+            torch.cuda.set_device(local_rank)
+            dist.init_process_group(backend=backend, rank=rank, world_size=world,
+                                    device_id=torch.device("cuda", local_rank))
+        else:
+            dist.init_process_group(backend=backend, rank=rank, world_size=world)
     return rank, local_rank, world
 
 
