@@ -13,6 +13,11 @@
 //                      once per stage that the sum stayed in range (see Online), so the common
 //                      case is one exponential and no comparison per logit.
 //   verify_rows_plain  one CTA per item with scalar global loads; any alignment.  Fallback.
+//
+// The same streaming kernel with a running arg max serves the greedy decoding step (Eq. 6),
+// and with a closing kernel that leaves (maximum, sum, draft logit) per row instead of the
+// decision it serves an LLM head whose columns are split over several ranks (ssd_verify_shard,
+// ssd_verify_combine).
 #include <limits.h>
 #include <math.h>
 

@@ -5,13 +5,14 @@
 //
 // Rows are visited position-major (position 0 of every utterance, then position 1, ...), claimed
 // in that order by persistent CTAs from a global counter, so that all CTAs work on about the
-// same position at any time and stay equally loaded although rows drop out at random.  A row is finalised inside the streaming kernel: the consumer warps leave their
-// (reference, sum) pairs and the draft token's logit in shared memory, and the producer warp,
-// when it is about to refill the stage that held the row's last part, merges them, writes the
-// row's log-likelihood and, on a reject, lowers the utterance's first-reject word in global
-// memory with an atomic minimum.  Before a row is fetched the producer reads that word and
-// skips the row if a smaller rejected position is already known.  Positions up to the true
-// first reject are therefore never skipped, and the result is exactly that of ssd_verify.
+// same position at any time and stay equally loaded although rows drop out at random.  A row
+// is finalised inside the streaming kernel: the consumer warps leave their (reference, sum)
+// pairs and the draft token's logit in shared memory, and the producer warp, when it is about
+// to refill the stage that held the row's last part, merges them, writes the row's
+// log-likelihood and, on a reject, lowers the utterance's first-reject word in global memory
+// with an atomic minimum.  Before a row is fetched the producer reads that word and skips the
+// row if a smaller rejected position is already known.  Positions up to the true first reject
+// are therefore never skipped, and the result is exactly that of ssd_verify.
 #include <limits.h>
 #include <math.h>
 
