@@ -138,10 +138,10 @@ __global__ void __launch_bounds__(544, 1) verify_rows_ee(const EeParams p) {
         bool failed = false;
         const int max_chunks = p.stage_bytes >> 4;
 
-        // Merges the partials of the row whose last part stage `st` held, once the consumers
-        // have let go of that stage; called by all lanes right after the stage's empty wait.
-        auto finalize = [&](int st) {
-            const int slot1 = pending[st];
+        // Merges the partials of the row in row slot slot1 - 1 (0: none), once the consumers
+        // have let go of the stage that held its last part; called by all lanes.  It touches
+        // the row slot only, not the stage, so it runs after the stage's next copy is under way.
+        auto finalize = [&](int slot1) {
             if (slot1 == 0) return;
             const int slot = slot1 - 1;
             const float2 v = lane < CW ? spart[slot * CW + lane] : make_float2(kNegInit, 0.f);
@@ -168,7 +168,6 @@ __global__ void __launch_bounds__(544, 1) verify_rows_ee(const EeParams p) {
                 if (fl) atomicOr(&p.flags[rm.b], fl);
                 if (reject) atomicMin(&p.first_reject[rm.b], rm.pos);
                 atomicAdd(&p.rows_read[rm.b], 1);
-                pending[st] = 0;
             }
             __syncwarp();
         };
@@ -238,7 +237,8 @@ __global__ void __launch_bounds__(544, 1) verify_rows_ee(const EeParams p) {
                 }
                 for (int part = 0; part < parts; ++part) {
                     if (!mbar_wait_bounded(empty0 + s * 8, ph ^ 1u)) { failed = true; break; }
-                    finalize(s);
+                    const int done_slot1 = pending[s];     // the row this stage held last, if any
+                    __syncwarp();
                     const int pc0 = part * per_part;
                     const int pc1 = min(row_chunks, pc0 + per_part);
                     const ranges::PartReads pr = ranges::part_reads(geom, pc0, pc1);
@@ -289,6 +289,7 @@ __global__ void __launch_bounds__(544, 1) verify_rows_ee(const EeParams p) {
                         }
                     }
                     __syncwarp();
+                    finalize(done_slot1);
                     if (++s == S) { s = 0; ph ^= 1u; }
                 }
             }
@@ -296,7 +297,7 @@ __global__ void __launch_bounds__(544, 1) verify_rows_ee(const EeParams p) {
         if (!failed) {
             // end marker into the next stage, then the rows still waiting in the other stages
             if (mbar_wait_bounded(empty0 + s * 8, ph ^ 1u)) {
-                finalize(s);
+                finalize(pending[s]);
                 if (lane == 0) {
                     desc[s].nchunks = 0; desc[s].flags = kFlagEnd; desc[s].slot = 0; desc[s].gather = -1;
                     mbar_arrive(full0 + s * 8);
@@ -304,7 +305,7 @@ __global__ void __launch_bounds__(544, 1) verify_rows_ee(const EeParams p) {
                 for (int t = 1; t < S && !failed; ++t) {
                     const int st = (s + t) % S;
                     const uint32_t par = st > s ? (ph ^ 1u) : ph;     // filled last round / this round
-                    if (mbar_wait_bounded(empty0 + st * 8, par)) finalize(st);
+                    if (mbar_wait_bounded(empty0 + st * 8, par)) finalize(pending[st]);
                     else failed = true;
                 }
             } else {
