@@ -58,6 +58,9 @@ def parse_args():
     ap.add_argument("--sweep-filter", default="", help="only points whose name contains this")
     ap.add_argument("--ncu-small", action="store_true",
                     help="profiling aid: one input set, no end-to-end leg, no CPU baseline")
+    ap.add_argument("--ring-sweep", action="store_true",
+                    help="time ssd_verify's streaming kernel on --config for several stage sizes "
+                         "of its shared-memory ring (one JSON line each) instead of the benchmark")
     ap.add_argument("--ncu-stage1", action="store_true",
                     help="profiling aid: only the CTC batch of --config (a fraction of a GB even "
                          "where the whole step holds tens), ssd_ctc_draft three times, no timing")
@@ -767,10 +770,55 @@ def run_stage1_only(args):
                       "dtype": w.dtype, "calls": 3}))
 
 
+def run_ring_sweep(args):
+    """ssd_verify's streaming kernel against the stage size of its ring (launch option
+    stage_bytes; 0 = the library's own choice): CUDA events the library records around the
+    kernel, rotating input sets, mean of 40 launches after 6 warm-up ones."""
+    import torch
+    from paper_2603_11243_b200 import binding as ssd
+    from paper_2603_11243_b200 import build as lib_build
+    from paper_2603_11243_b200 import synth
+    lib_build.build()
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    w = synth.CONFIGS[args.config]
+    sets = build_sets(w, device, N_SETS)
+    code = ssd.BF16 if w.dtype == "bf16" else ssd.F32
+    row_bytes = w.V_llm * (2 if w.dtype == "bf16" else 4)
+    for sb in (0, 16512, 24704, 32896, 49280, 65536, 98432):
+        o = ssd.LaunchOpts()
+        o.stage_bytes = sb
+        try:
+            outs = [ssd.alloc_verify_outputs(s["M"], s["B"], device,
+                                             ssd.ssd_verify_workspace_bytes(s["B"], s["M"], w.V_llm, code, o))
+                    for s in sets]
+            n = 40
+            ev = make_events(2 * n)
+            for it in range(n + 6):
+                s = sets[it % len(sets)]
+                if it >= 6:
+                    o.ev_begin, o.ev_end = ev[2 * (it - 6)].cuda_event, ev[2 * (it - 6) + 1].cuda_event
+                ssd.ssd_verify(s["vb"].logits, s["tok_off"], s["ids"], w.tau_slm,
+                               skip=s["gate"]["gate_accept"], out=outs[it % len(sets)], opts=o)
+            torch.cuda.synchronize()
+        except ssd.SsdError as e:
+            print(json.dumps({"stage_bytes": sb, "refused": str(e)}), flush=True)
+            continue
+        us = statistics.mean(ev[2 * i].elapsed_time(ev[2 * i + 1]) for i in range(n)) * 1e3
+        nbytes = statistics.mean(s["verify_bytes"] for s in sets)
+        stages_per_row = None if sb == 0 else -(-(row_bytes + 32) // sb)
+        print(json.dumps({"workload": w.name, "stage_bytes": sb or "library default",
+                          "stages_per_row": stages_per_row, "kernel_us": round(us, 1),
+                          "gbs": round(nbytes / (us * 1e-6) / 1e9, 1)}), flush=True)
+
+
 def main():
     args = parse_args()
     if args.sweep:
         run_sweep(args)
+        return
+    if args.ring_sweep:
+        run_ring_sweep(args)
         return
     if args.ncu_stage1:
         run_stage1_only(args)
