@@ -67,14 +67,17 @@ typedef struct ssd_launch_opts {
     int32_t kernel;       /* 0 auto; 1 plain-load kernels; 2 bulk-copy (TMA) pipelined kernels */
     int32_t ctas;         /* grid size of the streaming kernel */
     int32_t warps;        /* compute warps per CTA of the streaming kernel */
-    int32_t stages;       /* shared-memory pipeline depth */
-    int32_t stage_bytes;  /* bytes per pipeline stage (verify) / rows per stage (ctc_draft) */
-    int32_t split;        /* verify: column spans per logits row */
+    int32_t stages;       /* verify: shared-memory pipeline depth */
+    int32_t stage_bytes;  /* bytes per pipeline stage (verify) / passes per tile (ctc_draft) */
+    int32_t split;        /* verify: column spans per logits row; ctc_draft: lanes per row
+                             (2, 4, 8, 16 or 32; refused with SSD_ERR_ARG when a lane would walk
+                             more than 160 16-byte chunks of a row) */
     void *ev_begin;       /* cudaEvent_t recorded just before the streaming kernel, or NULL */
     void *ev_end;         /* cudaEvent_t recorded just after the streaming kernel, or NULL */
-    int32_t fma_exp;      /* verify, bf16: pairs of exponentials per 16-byte chunk evaluated by a
+    int32_t fma_exp;      /* bf16: pairs of exponentials per 16-byte chunk evaluated by a
                              polynomial on the FMA pipe instead of the special-function unit:
-                             0 auto; 1..3 that many of the 4 pairs; -1 none */
+                             0 auto; 1..3 that many of the 4 pairs (ctc_draft: at most 2);
+                             -1 none */
 } ssd_launch_opts;
 
 /* Human-readable name of a return code (static storage). */
@@ -114,8 +117,12 @@ size_t ssd_verify_workspace_bytes(int32_t B, int64_t M, int32_t V, ssd_dtype dty
  * draft_tokens   [N] i32 (U <= T guarantees the capacity; entries past draft_len[b] inside an
  *                utterance's range are left untouched)
  * draft_len, draft_full_len [B] i32   utt_max_entropy [B] f32   utt_status [B] u32 (overwritten)
- * workspace      at least ssd_ctc_draft_workspace_bytes(...) bytes, 256-byte aligned; may be
- *                NULL when that is 0.
+ * workspace      NULL, or at least ssd_ctc_draft_workspace_bytes(...) bytes (2,048), 256-byte
+ *                aligned: counters from which the streaming kernel's warps claim their tiles
+ *                of frames, so that SMs that run ahead take more.  It needs no clearing, before
+ *                the first call or between calls (the words carry a per-call tag), but two
+ *                calls whose kernels may run at the same time must not share it.  Without it
+ *                the tiles are dealt out in a fixed order; the results are the same.
  * Errors: SSD_ERR_NULL, SSD_ERR_ARG (B,N < 0; V < 1; ld < V; blank_id outside [0,V);
  * max_draft_len < 0), SSD_ERR_DTYPE, SSD_ERR_ALIGN, SSD_ERR_WORKSPACE, SSD_ERR_CUDA.
  */
@@ -137,12 +144,21 @@ int32_t ssd_ctc_draft(const void *logits, ssd_dtype dtype, int32_t V, int64_t ld
  *                                     a NaN entropy or malformed offsets never pass)
  *   max_entropy[b]  = max over the utterance's frames (0 if none)
  *   argmax_frame[b] = first frame attaining it, -1 if none                     (nullable)
- * frame_entropy [N] f32 may come from ssd_ctc_draft or anywhere else.
+ * Two forms:
+ *   from frame entropies   utt_max_entropy == NULL (or argmax_frame wanted): frame_entropy [N]
+ *                          f32, from ssd_ctc_draft or anywhere else, is read once;
+ *   from utterance maxima  utt_max_entropy [B] f32 and utt_status [B] u32 as ssd_ctc_draft left
+ *                          them, argmax_frame == NULL: "all frames below tau" is "the maximum is
+ *                          below tau", so B values are read instead of N (frame_entropy and
+ *                          frame_off are not looked at and may be NULL); an utterance whose
+ *                          status has SSD_UTT_NONFINITE, SSD_UTT_BAD_OFFSETS or SSD_UTT_INTERNAL
+ *                          set does not pass, exactly as in the first form.
  * Errors: SSD_ERR_NULL, SSD_ERR_ARG, SSD_ERR_CUDA.
  */
 int32_t ssd_entropy_gate(const float *frame_entropy, const int64_t *frame_off,
                          int32_t B, int64_t N, float tau_ctc,
                          uint8_t *gate_accept, float *max_entropy, int32_t *argmax_frame,
+                         const float *utt_max_entropy, const uint32_t *utt_status,
                          void *stream);
 
 /*

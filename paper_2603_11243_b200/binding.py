@@ -60,7 +60,7 @@ def lib():
                                     vp, vp, vp, vp, vp, vp, vp, vp, vp, vp,
                                     vp, C.c_size_t, vp, vp]
         L.ssd_entropy_gate.restype = i32
-        L.ssd_entropy_gate.argtypes = [vp, vp, i32, i64, C.c_float, vp, vp, vp, vp]
+        L.ssd_entropy_gate.argtypes = [vp, vp, i32, i64, C.c_float, vp, vp, vp, vp, vp, vp]
         L.ssd_verify.restype = i32
         L.ssd_verify.argtypes = [vp, C.c_int, i32, i64, vp, vp, i32, i64, C.c_float, vp,
                                  vp, vp, vp, vp, vp, vp, C.c_size_t, vp, vp]
@@ -163,7 +163,9 @@ def ssd_verify_read_span(base_addr: int, dtype_code: int, V: int, ld: int, M: in
 
 def alloc_ctc_outputs(N: int, B: int, device, logprob_ld: int = 0) -> Dict[str, torch.Tensor]:
     e = lambda n, dt: torch.empty((n,), dtype=dt, device=device)
-    out = dict(frame_entropy=e(N, torch.float32), frame_argmax=e(N, torch.int32),
+    # ssd_ctc_draft_workspace_bytes is 2048 whatever the sizes are (the tile counters)
+    out = dict(workspace=torch.empty((2048,), dtype=torch.uint8, device=device),
+               frame_entropy=e(N, torch.float32), frame_argmax=e(N, torch.int32),
                frame_lse=e(N, torch.float32), draft_tokens=e(N, torch.int32),
                draft_frames=e(N, torch.int32), draft_len=e(B, torch.int32),
                draft_full_len=e(B, torch.int32), utt_max_entropy=e(B, torch.float32),
@@ -184,6 +186,7 @@ def ssd_ctc_draft(logits: torch.Tensor, frame_off: torch.Tensor, blank_id: int,
         raise TypeError("frame_off must be int64")
     if out is None:
         out = alloc_ctc_outputs(N, B, logits.device, ld if want_logprob else 0)
+    ws = out.get("workspace")
     rc = lib().ssd_ctc_draft(
         _dev(logits, "logits"), _dtype_code(logits), V, ld, _dev(frame_off, "frame_off"), B, N,
         blank_id, max_draft_len, _dev(out["frame_entropy"], "frame_entropy"),
@@ -192,7 +195,7 @@ def ssd_ctc_draft(logits: torch.Tensor, frame_off: torch.Tensor, blank_id: int,
         _dev(out["draft_tokens"], "draft_tokens"), _dev(out.get("draft_frames"), "draft_frames"),
         _dev(out["draft_len"], "draft_len"), _dev(out["draft_full_len"], "draft_full_len"),
         _dev(out["utt_max_entropy"], "utt_max_entropy"), _dev(out["utt_status"], "utt_status"),
-        None, 0, _stream(), _opts(opts))
+        _dev(ws, "workspace"), 0 if ws is None else ws.numel(), _stream(), _opts(opts))
     if rc != OK:
         raise SsdError(rc, "ssd_ctc_draft")
     return out
@@ -216,7 +219,31 @@ def ssd_entropy_gate(frame_entropy: torch.Tensor, frame_off: torch.Tensor, tau_c
         _dev(frame_entropy, "frame_entropy"), _dev(frame_off, "frame_off"), B, N,
         C.c_float(tau_ctc), _dev(out["gate_accept"], "gate_accept"),
         _dev(out["max_entropy"], "max_entropy"), _dev(out.get("argmax_frame"), "argmax_frame"),
-        _stream())
+        None, None, _stream())
+    if rc != OK:
+        raise SsdError(rc, "ssd_entropy_gate")
+    return out
+
+
+def _gate_from_maxima_args(utt_max_entropy, utt_status, tau_ctc, out):
+    B = utt_max_entropy.shape[0]
+    if utt_max_entropy.dtype != torch.float32 or utt_status.dtype != torch.int32:
+        raise TypeError("utt_max_entropy must be float32 and utt_status int32 (the bits of a uint32)")
+    return [None, None, B, 0, C.c_float(tau_ctc), _dev(out["gate_accept"], "gate_accept"),
+            _dev(out["max_entropy"], "max_entropy"), None,
+            _dev(utt_max_entropy, "utt_max_entropy"), _dev(utt_status, "utt_status"), _stream()]
+
+
+def ssd_entropy_gate_from_maxima(utt_max_entropy: torch.Tensor, utt_status: torch.Tensor,
+                                 tau_ctc: float, out=None) -> Dict[str, torch.Tensor]:
+    """The entropy gate (Eq. 3) through ssd_entropy_gate's second form: from the utterance
+    maxima and status words ssd_ctc_draft left behind (B values instead of N frame entropies).
+    `out` needs gate_accept and max_entropy only."""
+    if out is None:
+        B, dev = utt_max_entropy.shape[0], utt_max_entropy.device
+        out = dict(gate_accept=torch.empty((B,), dtype=torch.uint8, device=dev),
+                   max_entropy=torch.empty((B,), dtype=torch.float32, device=dev))
+    rc = lib().ssd_entropy_gate(*_gate_from_maxima_args(utt_max_entropy, utt_status, tau_ctc, out))
     if rc != OK:
         raise SsdError(rc, "ssd_entropy_gate")
     return out
@@ -510,7 +537,8 @@ def bind_ctc_draft(logits, frame_off, blank_id, max_draft_len, out, V=None,
             _dev(out.get("draft_frames"), "draft_frames"), _dev(out["draft_len"], "draft_len"),
             _dev(out["draft_full_len"], "draft_full_len"),
             _dev(out["utt_max_entropy"], "utt_max_entropy"), _dev(out["utt_status"], "utt_status"),
-            None, 0, _stream(), _opts(opts)]
+            _dev(out.get("workspace"), "workspace"),
+            0 if out.get("workspace") is None else out["workspace"].numel(), _stream(), _opts(opts)]
     return BoundCall(lib().ssd_ctc_draft, "ssd_ctc_draft", args, (logits, frame_off, out, opts), True)
 
 
@@ -519,9 +547,15 @@ def bind_entropy_gate(frame_entropy, frame_off, tau_ctc, out) -> BoundCall:
     args = [_dev(frame_entropy, "frame_entropy"), _dev(frame_off, "frame_off"), B, N,
             C.c_float(tau_ctc), _dev(out["gate_accept"], "gate_accept"),
             _dev(out["max_entropy"], "max_entropy"), _dev(out.get("argmax_frame"), "argmax_frame"),
-            _stream()]
+            None, None, _stream()]
     return BoundCall(lib().ssd_entropy_gate, "ssd_entropy_gate", args,
                      (frame_entropy, frame_off, out), False)
+
+
+def bind_entropy_gate_from_maxima(utt_max_entropy, utt_status, tau_ctc, out) -> BoundCall:
+    return BoundCall(lib().ssd_entropy_gate, "ssd_entropy_gate",
+                     _gate_from_maxima_args(utt_max_entropy, utt_status, tau_ctc, out),
+                     (utt_max_entropy, utt_status, out), False)
 
 
 def bind_verify(logits, tok_off, draft_ids, tau_slm, out, skip=None, V=None,

@@ -32,8 +32,10 @@ int32_t ssd_version(void) { return 100; }
 
 size_t ssd_ctc_draft_workspace_bytes(int32_t B, int64_t N, int32_t V, ssd_dtype dtype,
                                      const ssd_launch_opts *opts) {
-    (void)B; (void)N; (void)V; (void)dtype; (void)opts;
-    return 0;
+    if (B < 0 || N < 0 || V < 1 || (dtype != SSD_F32 && dtype != SSD_BF16)) return 0;
+    CtcPlan plan;
+    if (plan_ctc(dtype, V, V, N, B, opts, &plan) != SSD_OK) return 0;
+    return plan.workspace_bytes;
 }
 
 size_t ssd_verify_workspace_bytes(int32_t B, int64_t M, int32_t V, ssd_dtype dtype,
@@ -54,7 +56,6 @@ int32_t ssd_ctc_draft(const void *logits, ssd_dtype dtype, int32_t V, int64_t ld
                       float *utt_max_entropy, uint32_t *utt_status,
                       void *workspace, size_t workspace_bytes, void *stream,
                       const ssd_launch_opts *opts) {
-    (void)workspace; (void)workspace_bytes;
     if (dtype != SSD_F32 && dtype != SSD_BF16) return SSD_ERR_DTYPE;
     if (B < 0 || N < 0 || V < 1 || ld < V || blank_id < 0 || blank_id >= V || max_draft_len < 0)
         return SSD_ERR_ARG;
@@ -64,9 +65,15 @@ int32_t ssd_ctc_draft(const void *logits, ssd_dtype dtype, int32_t V, int64_t ld
         return SSD_ERR_NULL;
     const int es = dtype == SSD_F32 ? 4 : 2;
     if (reinterpret_cast<uintptr_t>(logits) % es) return SSD_ERR_ALIGN;
+    CtcPlan plan;
+    int rc = plan_ctc(dtype, V, ld, N, B, opts, &plan);
+    if (rc != SSD_OK) return rc;
+    if (workspace && (workspace_bytes < plan.workspace_bytes ||
+                      reinterpret_cast<uintptr_t>(workspace) % 256))
+        return SSD_ERR_WORKSPACE;
     Launch L{static_cast<cudaStream_t>(stream), opts};
-    int rc = launch_ctc_rows(logits, dtype, V, ld, N, frame_off, B, frame_entropy, frame_argmax,
-                             frame_lse, frame_logprob, utt_status, L);
+    rc = launch_ctc_rows(logits, dtype, V, ld, N, frame_entropy, frame_argmax, frame_lse,
+                         frame_logprob, workspace, plan, L);
     if (rc != SSD_OK) return rc;
     return launch_collapse(frame_argmax, frame_entropy, frame_off, B, N, blank_id, max_draft_len,
                            draft_tokens, draft_frames, draft_len, draft_full_len,
@@ -76,11 +83,18 @@ int32_t ssd_ctc_draft(const void *logits, ssd_dtype dtype, int32_t V, int64_t ld
 int32_t ssd_entropy_gate(const float *frame_entropy, const int64_t *frame_off,
                          int32_t B, int64_t N, float tau_ctc,
                          uint8_t *gate_accept, float *max_entropy, int32_t *argmax_frame,
+                         const float *utt_max_entropy, const uint32_t *utt_status,
                          void *stream) {
     if (B < 0 || N < 0) return SSD_ERR_ARG;
+    if (B > 0 && (!gate_accept || !max_entropy)) return SSD_ERR_NULL;
+    if (utt_max_entropy && !argmax_frame) {
+        // the maxima are already there: B values to look at instead of N
+        if (B > 0 && !utt_status) return SSD_ERR_NULL;
+        return launch_gate_from_maxima(utt_max_entropy, utt_status, B, tau_ctc, gate_accept,
+                                       max_entropy, static_cast<cudaStream_t>(stream));
+    }
     if (!frame_off) return SSD_ERR_NULL;
     if (N > 0 && !frame_entropy) return SSD_ERR_NULL;
-    if (B > 0 && (!gate_accept || !max_entropy)) return SSD_ERR_NULL;
     return launch_gate(frame_entropy, frame_off, B, N, tau_ctc, gate_accept, max_entropy,
                        argmax_frame, static_cast<cudaStream_t>(stream));
 }

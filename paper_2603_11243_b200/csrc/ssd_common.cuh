@@ -321,10 +321,21 @@ __device__ __forceinline__ int utterance_of_row(const int64_t *off, int B, int64
 }
 
 // ---- launchers implemented in the .cu files ---------------------------------------------------
+struct CtcPlan {
+    int kernel;          // 1 plain loads, 2 bulk-copy tiles
+    int lanes_per_row;   // G
+    int rows_per_tile;   // R
+    int warps, stages, stage_stride;
+    int iters, tail_from;   // chunk iterations per lane and row; first one that may be a row's last
+    int fma_exp;            // pairs per bf16 chunk whose exponential runs on the FMA pipe
+    int64_t num_tiles;
+    size_t smem_bytes, workspace_bytes;
+};
+int plan_ctc(ssd_dtype dtype, int V, int64_t ld, int64_t N, int B, const ssd_launch_opts *opts,
+             CtcPlan *plan);
 int launch_ctc_rows(const void *logits, ssd_dtype dtype, int V, int64_t ld, int64_t N,
-                    const int64_t *frame_off, int B, float *frame_entropy, int32_t *frame_argmax,
-                    float *frame_lse, float *frame_logprob, uint32_t *utt_status,
-                    const Launch &L);
+                    float *frame_entropy, int32_t *frame_argmax, float *frame_lse,
+                    float *frame_logprob, void *workspace, const CtcPlan &plan, const Launch &L);
 int launch_collapse(const int32_t *frame_argmax, const float *frame_entropy,
                     const int64_t *frame_off, int B, int64_t N, int blank_id, int max_draft_len,
                     int32_t *draft_tokens, int32_t *draft_frames, int32_t *draft_len,
@@ -333,16 +344,9 @@ int launch_collapse(const int32_t *frame_argmax, const float *frame_entropy,
 int launch_gate(const float *frame_entropy, const int64_t *frame_off, int B, int64_t N,
                 float tau, uint8_t *gate_accept, float *max_entropy, int32_t *argmax_frame,
                 cudaStream_t stream);
-
-struct CtcPlan {
-    int kernel;          // 1 plain loads, 2 bulk-copy tiles
-    int lanes_per_row;   // G
-    int rows_per_tile;   // R
-    int warps, stages, stage_stride;
-    int64_t num_tiles;
-};
-int plan_ctc(ssd_dtype dtype, int V, int64_t ld, int64_t N, const ssd_launch_opts *opts,
-             CtcPlan *plan);
+int launch_gate_from_maxima(const float *utt_max_entropy, const uint32_t *utt_status, int B,
+                            float tau, uint8_t *gate_accept, float *max_entropy,
+                            cudaStream_t stream);
 
 struct VerifyPlan {
     int kernel;        // 1 plain loads, 2 bulk-copy pipeline

@@ -2,11 +2,13 @@
 // B of Section 2.1, and the entropy gate of Eq. 3.
 //
 // Frame statistics are one streaming read of the [N, V] logits.  Two kernels compute them:
-//   ctc_rows_tma    each warp owns a small ring of shared-memory stages that it fills with 1-D
-//                   bulk asynchronous copies (TMA) of a few consecutive rows and drains itself:
-//                   no block-level synchronisation at all.  A row sits in shared memory while it
-//                   is reduced, so the exact two-pass softmax (max, then exponentials) costs one
-//                   HBM read and one exponential per logit.
+//   ctc_rows_tma    each warp owns a shared-memory stage that it fills with one 1-D bulk
+//                   asynchronous copy (TMA) of a few consecutive rows and drains itself: no
+//                   block-level synchronisation after set-up.  G lanes share a row; one fused
+//                   pass per row keeps a running maximum and the sums of 2^t and t*2^t
+//                   relative to a per-lane reference, so a logit costs one exponential; rows
+//                   that pass cannot take (masked -inf logits, NaN, +inf, a range beyond fp32)
+//                   are redone from shared memory by an exact two-pass routine.
 //   ctc_rows_plain  one warp per row with scalar global loads; any alignment, any V.  Fallback.
 #include <limits.h>
 #include <math.h>
@@ -31,41 +33,44 @@ struct CtcParams {
     int stages;
     int stage_stride;      // bytes, multiple of 128
     int warps;
+    int iters;             // chunk iterations per lane and row: ceil(most chunks a row touches / G)
+    int tail_from;         // first iteration (>= 1) in which a lane may meet its row's last chunk
     float *frame_entropy;
     int32_t *frame_argmax;
     float *frame_lse;
     float *frame_logprob;
+    // tiles are handed out from kTileCounters counters in the caller's workspace, 256 bytes
+    // apart (NULL: tile j to warp j mod the number of warps).  A word is {epoch : 32 | count :
+    // 32}, so a call needs no clearing of what the last one left there.
+    unsigned long long *tile_counter;
+    uint32_t epoch;
+    int counters;          // C
+    int claim;             // tiles per claim
 };
+constexpr int kTileCounters = 4;      // at most; a launch uses the largest divisor of its warps per CTA
 
 // Replaces the elements of a 16-byte chunk outside [e_lo, e_hi) (they belong to a neighbouring
-// row, to the padding between rows, or were never written) by -inf, or, with kFinite, by a
-// finite value near -1e30 whose exponential is 0 and whose product with that 0 is not NaN.
-template <typename T, bool kFinite>
-__device__ __forceinline__ void mask_chunk(uint4 &w, int e_lo, int e_hi);
-template <bool kFinite> __device__ __forceinline__ void mask_f32(uint4 &w, int e_lo, int e_hi) {
-    const uint32_t fill = kFinite ? 0xf149f2cau : 0xff800000u;
+// row, to the padding between rows, or were never written) by -inf.
+template <typename T> __device__ __forceinline__ void mask_chunk(uint4 &w, int e_lo, int e_hi);
+template <> __device__ __forceinline__ void mask_chunk<float>(uint4 &w, int e_lo, int e_hi) {
+    const uint32_t fill = 0xff800000u;
     if (0 < e_lo || 0 >= e_hi) w.x = fill;
     if (1 < e_lo || 1 >= e_hi) w.y = fill;
     if (2 < e_lo || 2 >= e_hi) w.z = fill;
     if (3 < e_lo || 3 >= e_hi) w.w = fill;
 }
-template <bool kFinite>
 __device__ __forceinline__ uint32_t mask_pair(uint32_t v, int j, int e_lo, int e_hi) {
-    const uint32_t fill = kFinite ? 0xf149u : 0xff80u;
+    const uint32_t fill = 0xff80u;
     if (j < e_lo || j >= e_hi) v = (v & 0xffff0000u) | fill;
     if (j + 1 < e_lo || j + 1 >= e_hi) v = (v & 0x0000ffffu) | (fill << 16);
     return v;
 }
-template <bool kFinite> __device__ __forceinline__ void mask_bf16(uint4 &w, int e_lo, int e_hi) {
-    w.x = mask_pair<kFinite>(w.x, 0, e_lo, e_hi);
-    w.y = mask_pair<kFinite>(w.y, 2, e_lo, e_hi);
-    w.z = mask_pair<kFinite>(w.z, 4, e_lo, e_hi);
-    w.w = mask_pair<kFinite>(w.w, 6, e_lo, e_hi);
+template <> __device__ __forceinline__ void mask_chunk<bf16_t>(uint4 &w, int e_lo, int e_hi) {
+    w.x = mask_pair(w.x, 0, e_lo, e_hi);
+    w.y = mask_pair(w.y, 2, e_lo, e_hi);
+    w.z = mask_pair(w.z, 4, e_lo, e_hi);
+    w.w = mask_pair(w.w, 6, e_lo, e_hi);
 }
-template <> __device__ __forceinline__ void mask_chunk<float, false>(uint4 &w, int a, int b) { mask_f32<false>(w, a, b); }
-template <> __device__ __forceinline__ void mask_chunk<float, true>(uint4 &w, int a, int b) { mask_f32<true>(w, a, b); }
-template <> __device__ __forceinline__ void mask_chunk<bf16_t, false>(uint4 &w, int a, int b) { mask_bf16<false>(w, a, b); }
-template <> __device__ __forceinline__ void mask_chunk<bf16_t, true>(uint4 &w, int a, int b) { mask_bf16<true>(w, a, b); }
 
 // S += 2^t, A += t * 2^t for the elements of one chunk, t = x*log2e - mh.  Elements are first
 // clamped from below so that a masked (-inf) logit gives t*2^t = 0 instead of NaN.
@@ -140,7 +145,7 @@ __device__ __noinline__ RowOut reduce_row_exact(uint32_t stage_addr, RowSpan r, 
     int vc = -1;
     for (int c = cf + sub; c <= cl; c += G) {
         uint4 w = lds128(stage_addr + (uint32_t)c * 16);
-        if (c == cf || c == cl) mask_chunk<T, false>(w, c == cf ? e_lo : 0, c == cl ? e_hi : EPC);
+        if (c == cf || c == cl) mask_chunk<T>(w, c == cf ? e_lo : 0, c == cl ? e_hi : EPC);
         const float cm = chunk_max<T>(w);
         if (cm > vmax) { vmax = cm; vc = c; }
     }
@@ -148,7 +153,7 @@ __device__ __noinline__ RowOut reduce_row_exact(uint32_t stage_addr, RowSpan r, 
     int cand = INT_MAX;
     if (vc >= 0 && vmax == m) {
         uint4 w = lds128(stage_addr + (uint32_t)vc * 16);
-        if (vc == cf || vc == cl) mask_chunk<T, false>(w, vc == cf ? e_lo : 0, vc == cl ? e_hi : EPC);
+        if (vc == cf || vc == cl) mask_chunk<T>(w, vc == cf ? e_lo : 0, vc == cl ? e_hi : EPC);
         float x[EPC];
         chunk_unpack<T>(w, x);
         int j = EPC - 1;
@@ -164,7 +169,7 @@ __device__ __noinline__ RowOut reduce_row_exact(uint32_t stage_addr, RowSpan r, 
     float2 Sa = make_float2(0.f, 0.f), Sb = Sa, Aa = Sa, Ab = Sa;
     for (int c = cf + sub; c <= cl; c += G) {
         uint4 w = lds128(stage_addr + (uint32_t)c * 16);
-        if (c == cf || c == cl) mask_chunk<T, false>(w, c == cf ? e_lo : 0, c == cl ? e_hi : EPC);
+        if (c == cf || c == cl) mask_chunk<T>(w, c == cf ? e_lo : 0, c == cl ? e_hi : EPC);
         entropy_chunk<T>(w, -mh, Sa, Sb, Aa, Ab);
     }
     const float S = group_sum<G>((Sa.x + Sa.y) + (Sb.x + Sb.y));
@@ -177,53 +182,145 @@ __device__ __noinline__ RowOut reduce_row_exact(uint32_t stage_addr, RowSpan r, 
     return out;
 }
 
-// One chunk of the fused pass: running maximum (with the chunk it was first met in) and the
-// sums S += 2^t, A += t*2^t with t = x*log2e - rh for a per-lane reference rh (in log2 units).
+// ---- the fused pass with a uniform trip count ---------------------------------------------------
+// Every lane makes the same number of chunk iterations per row (p.iters, fixed by V and G alone),
+// so a pass over 32/G rows has no data-dependent control flow.  Iteration 0 and the iterations
+// from p.tail_from on may meet a row's first or last chunk, or lie past the row's end: their
+// chunk goes through a keep mask looked up in a small shared-memory table (which elements
+// [lo, hi) of a chunk are the row's own; hi = 0 keeps nothing), and what is not kept becomes a
+// finite fill value near -1e30 whose exponential is 0.  The iterations in between are interior
+// chunks and take no mask at all.
+template <typename T> struct FillWord;
+template <> struct FillWord<float> { static constexpr uint32_t v = 0xf149f2cau; };
+template <> struct FillWord<bf16_t> { static constexpr uint32_t v = 0xf149f149u; };
+
+// table entry (lo, hi) at index lo * (EPC + 1) + hi: all-ones in the bytes of elements [lo, hi)
 template <typename T>
-__device__ __forceinline__ void fused_chunk(const uint4 &w, int c, float nrh, float &vmax, int &vc,
-                                            float2 &Sa, float2 &Sb, float2 &Aa, float2 &Ab);
-template <>
-__device__ __forceinline__ void fused_chunk<float>(const uint4 &w, int c, float nrh, float &vmax,
-                                                   int &vc, float2 &Sa, float2 &Sb, float2 &Aa,
-                                                   float2 &Ab) {
-    const float cm = chunk_max<float>(w);
-    if (cm > vmax) { vmax = cm; vc = c; }
-    entropy_pair(make_float2(__uint_as_float(w.x), __uint_as_float(w.y)), nrh, Sa, Aa);
-    entropy_pair(make_float2(__uint_as_float(w.z), __uint_as_float(w.w)), nrh, Sb, Ab);
-}
-template <>
-__device__ __forceinline__ void fused_chunk<bf16_t>(const uint4 &w, int c, float nrh, float &vmax,
-                                                    int &vc, float2 &Sa, float2 &Sb, float2 &Aa,
-                                                    float2 &Ab) {
-    const float cm = chunk_max<bf16_t>(w);
-    if (cm > vmax) { vmax = cm; vc = c; }
-    entropy_pair(make_float2(bf16_lo(w.x), bf16_hi(w.x)), nrh, Sa, Aa);
-    entropy_pair(make_float2(bf16_lo(w.y), bf16_hi(w.y)), nrh, Sb, Ab);
-    entropy_pair(make_float2(bf16_lo(w.z), bf16_hi(w.z)), nrh, Sa, Aa);
-    entropy_pair(make_float2(bf16_lo(w.w), bf16_hi(w.w)), nrh, Sb, Ab);
+__device__ __forceinline__ void build_keep_table(uint4 *tab, int tid, int nthreads) {
+    constexpr int EPC = Elem<T>::kPerChunk, ES = Elem<T>::kBytes;
+    for (int e = tid; e < EPC * (EPC + 1); e += nthreads) {
+        const int lo = e / (EPC + 1), hi = e - lo * (EPC + 1);
+        uint32_t k[4];
+#pragma unroll
+        for (int wd = 0; wd < 4; ++wd) {
+            if (ES == 4) {
+                k[wd] = (lo <= wd && wd < hi) ? 0xffffffffu : 0u;
+            } else {
+                k[wd] = ((lo <= 2 * wd && 2 * wd < hi) ? 0x0000ffffu : 0u) |
+                        ((lo <= 2 * wd + 1 && 2 * wd + 1 < hi) ? 0xffff0000u : 0u);
+            }
+        }
+        tab[e] = make_uint4(k[0], k[1], k[2], k[3]);
+    }
 }
 
-// Frame statistics of the rows of one tile that lies in shared memory.  G lanes share a row
-// and a warp works on 32/G rows at a time.  A row is walked in the 16-byte chunks of the stage
-// (whose alignment is that of global memory); its first and last chunk may also hold foreign
-// elements, which are masked.
+template <typename T> __device__ __forceinline__ uint4 lds_keep(uint32_t addr, uint32_t entry) {
+    constexpr uint32_t F = FillWord<T>::v;
+    uint4 w = lds128(addr);
+    const uint4 k = lds128(entry);
+    w.x = (w.x & k.x) | (F & ~k.x);
+    w.y = (w.y & k.y) | (F & ~k.y);
+    w.z = (w.z & k.z) | (F & ~k.z);
+    w.w = (w.w & k.w) | (F & ~k.w);
+    return w;
+}
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
+// 2^t for a pair on the FMA pipe, for t already known to be >= -126 (the caller clamps the
+// logits from below) and not checked from above (the caller tests its largest exponent once
+// per row): nearest integer n by the 1.5*2^23 trick, a degree-4 polynomial for 2^f on
+// f = t - n in [-1/2, 1/2] (relative error 3.6e-6), n added into the exponent field.
+__device__ __forceinline__ float2 exp2_fma_pair_inrange(float2 t) {
+    const float kMagic = 12582912.f;
+    const float2 r = fadd2(t, make_float2(kMagic, kMagic));
+    const float2 n = fadd2(r, make_float2(-kMagic, -kMagic));
+    const float2 f = ffma2(n, make_float2(-1.f, -1.f), t);
+    float2 q = make_float2(0.00966636836528778f, 0.00966636836528778f);
+    q = ffma2(q, f, make_float2(0.055921975523233414f, 0.055921975523233414f));
+    q = ffma2(q, f, make_float2(0.2402234971523285f, 0.2402234971523285f));
+    q = ffma2(q, f, make_float2(0.6931210160255432f, 0.6931210160255432f));
+    q = ffma2(q, f, make_float2(1.0f, 1.0f));
+    float2 y;
+    y.x = __int_as_float(__float_as_int(r.x) * (1 << 23) + __float_as_int(q.x));
+    y.y = __int_as_float(__float_as_int(r.y) * (1 << 23) + __float_as_int(q.y));
+    return y;
+}
+
+// S += 2^t, A += t*2^t over one chunk (t = x*log2e + nrh) and the running maximum with the
+// chunk it was first met in.  With kF, that many of a bf16 chunk's four pairs take the FMA-pipe
+// exponential; `floor2` is then a packed pair of a bf16 value below which those logits are
+// raised first (their exponentials are below 2^-124 either way).
+template <int kF> __device__ __forceinline__ void entropy_pair2(float2 x, float nrh, float2 &S, float2 &A) {
+    const float2 t = ffma2(x, make_float2(kLog2e, kLog2e), make_float2(nrh, nrh));
+    const float2 e = kF ? exp2_fma_pair_inrange(t) : make_float2(ex2(t.x), ex2(t.y));
+    S = fadd2(S, e);
+    A = ffma2(t, e, A);
+}
+template <typename T, int kF> struct FusedChunk;
+template <int kF> struct FusedChunk<float, kF> {
+    static __device__ __forceinline__ void run(const uint4 &w, int c, float nrh, uint32_t, float &vmax,
+                                               int &vc, float2 &Sa, float2 &Sb, float2 &Aa, float2 &Ab) {
+        const float x0 = __uint_as_float(w.x), x1 = __uint_as_float(w.y);
+        const float x2 = __uint_as_float(w.z), x3 = __uint_as_float(w.w);
+        const float nm = max3(max3(vmax, x0, x1), x2, x3);
+        if (nm > vmax) vc = c;
+        vmax = nm;
+        entropy_pair2<0>(make_float2(x0, x1), nrh, Sa, Aa);
+        entropy_pair2<0>(make_float2(x2, x3), nrh, Sb, Ab);
+    }
+};
+template <int kF> struct FusedChunk<bf16_t, kF> {
+    static __device__ __forceinline__ void run(const uint4 &w, int c, float nrh, uint32_t floor2,
+                                               float &vmax, int &vc, float2 &Sa, float2 &Sb,
+                                               float2 &Aa, float2 &Ab) {
+        const float x0 = bf16_lo(w.x), x1 = bf16_hi(w.x), x2 = bf16_lo(w.y), x3 = bf16_hi(w.y);
+        const float x4 = bf16_lo(w.z), x5 = bf16_hi(w.z), x6 = bf16_lo(w.w), x7 = bf16_hi(w.w);
+        const float nm = max3(max3(max3(max3(vmax, x0, x1), x2, x3), x4, x5), x6, x7);
+        if (nm > vmax) vc = c;
+        vmax = nm;
+        if (kF >= 1) {
+            const uint32_t u = bf16x2_max_nan(w.x, floor2);
+            entropy_pair2<1>(make_float2(bf16_lo(u), bf16_hi(u)), nrh, Sa, Aa);
+        } else {
+            entropy_pair2<0>(make_float2(x0, x1), nrh, Sa, Aa);
+        }
+        if (kF >= 2) {
+            const uint32_t u = bf16x2_max_nan(w.y, floor2);
+            entropy_pair2<1>(make_float2(bf16_lo(u), bf16_hi(u)), nrh, Sb, Ab);
+        } else {
+            entropy_pair2<0>(make_float2(x2, x3), nrh, Sb, Ab);
+        }
+        entropy_pair2<0>(make_float2(x4, x5), nrh, Sa, Aa);
+        entropy_pair2<0>(make_float2(x6, x7), nrh, Sb, Ab);
+    }
+};
+
+// Frame statistics of the rows of one tile that lies in shared memory.  G lanes share a row and
+// a warp works on 32/G rows at a time; a row is walked in the 16-byte chunks of the stage (whose
+// alignment is that of global memory), lane `sub` taking chunks sub, sub + G, ...
 //
 // Fused single pass: a lane takes the largest element of its first chunk as reference (rh =
 // fl(ref*log2e), in log2 units) and, for every chunk, updates its running maximum and adds 2^t
 // and t*2^t, t = x*log2e - rh (one fma).  fp32 keeps full relative precision whatever the
-// reference, so the sums only have to stay in range; at the end the lanes' sums are re-based
-// to mh = fl(m*log2e) of the row maximum m (S' = S*2^d, A' = (A + d*S)*2^d with d = rh - mh,
-// an exact difference) and added; ml = m*log2e - mh (exact, by fma) is taken out of the
-// log-sum-exp and cancels in the entropy.  One exponential per logit, and
-// the comparisons overlap with the exponentials.  A group whose sums left the range or turned
-// NaN (a logit far above the reference, masked -inf logits, NaN, +inf) is redone by the exact
-// two-pass routine above.
-template <typename T, int G>
-__device__ __forceinline__ void reduce_tile(const CtcParams &p, uint32_t stage_addr, uint32_t head,
-                                            int64_t r0, int nrows, int lane) {
+// reference, so the sums only have to stay in range; at the end the lanes' sums are re-based to
+// mh = fl(m*log2e) of the row maximum m (S' = S*2^d, A' = (A + d*S)*2^d with d = rh - mh, an
+// exact difference) and added; ml = m*log2e - mh (exact, by fma) is taken out of the log-sum-exp
+// and cancels in the entropy.  One exponential per logit.  A group whose sums left the range or
+// turned NaN (a logit far above the reference, masked -inf logits, NaN, +inf) is redone by the
+// exact two-pass routine above.
+template <typename T, int G, int kF>
+__device__ __forceinline__ void reduce_tile(const CtcParams &p, uint32_t stage_addr, uint32_t keep_tab,
+                                            uint32_t head, int64_t r0, int nrows, int lane) {
     constexpr int ES = Elem<T>::kBytes, EPC = Elem<T>::kPerChunk, RPW = 32 / G;
+    constexpr uint32_t STEP = (uint32_t)G * 16;
     const int sub = lane % G, grp = lane / G;
     const uint32_t pitch = (uint32_t)(p.ld * ES), row_bytes = (uint32_t)p.V * ES;
+    const int ITER = p.iters, KT = p.tail_from;
     for (int g0 = 0; g0 < nrows; g0 += RPW) {
         const int i = g0 + grp;
         const bool valid = i < nrows;
@@ -235,55 +332,89 @@ __device__ __forceinline__ void reduce_tile(const CtcParams &p, uint32_t stage_a
         r.e_hi = (int)((off + row_bytes - 1) & 15) / ES + 1;
         const int cf = r.cf, cl = r.cl;
 
-        float vmax = -INFINITY, ref = 0.f;
+        int c = cf + sub;
+        const bool has = c <= cl;
+        uint32_t a = stage_addr + (uint32_t)c * 16;
+        float vmax = -INFINITY;
         int vc = -1;
         float2 Sa = make_float2(0.f, 0.f), Sb = Sa, Aa = Sa, Ab = Sa;
-        int c = cf + sub;
-        if (c <= cl) {
-            // first chunk of this lane (an edge chunk for some lanes): fixes the reference
-            uint4 w = lds128(stage_addr + (uint32_t)c * 16);
-            if (c == cf || c == cl) mask_chunk<T, true>(w, c == cf ? r.e_lo : 0, c == cl ? r.e_hi : EPC);
+        float nrh;
+        uint32_t floor2 = 0;
+        bool coarse = false;
+        {
+            // iteration 0: the row's first chunk for lane 0 of the group (and, for a very short
+            // row, possibly its last one, or nothing at all)
+            const int lo = sub == 0 ? r.e_lo : 0;
+            const int hi = c < cl ? EPC : (c == cl ? r.e_hi : 0);
+            const uint4 w = lds_keep<T>(a, keep_tab + (uint32_t)(lo * (EPC + 1) + hi) * 16);
             const float cm = chunk_max<T>(w);
-            if (cm > -INFINITY) ref = cm * kLog2e;
-            fused_chunk<T>(w, c, -ref, vmax, vc, Sa, Sb, Aa, Ab);
-            c += G;
-#pragma unroll 2
-            for (; c < cl; c += G) {           // interior chunks: no masks
-                const uint4 wi = lds128(stage_addr + (uint32_t)c * 16);
-                fused_chunk<T>(wi, c, -ref, vmax, vc, Sa, Sb, Aa, Ab);
+            const float ref = cm > -1.0e29f ? cm : 0.f;
+            nrh = -(ref * kLog2e);
+            if (kF) {
+                // bf16 (rounded up) of ref - 85: t = (x - ref)*log2e stays above -126.  For
+                // |ref| < 4096 a bf16 step is at most 16, so the floor stays 69 below ref.
+                coarse = !(fabsf(ref) < 4096.f);
+                uint32_t fb = __float_as_uint(ref - 85.f);
+                fb = (fb & 0x80000000u) ? fb : fb + 0xffffu;
+                floor2 = (fb >> 16) * 0x10001u;
             }
-            if (c == cl) {                      // the row's last chunk
-                uint4 wl = lds128(stage_addr + (uint32_t)c * 16);
-                mask_chunk<T, true>(wl, 0, r.e_hi);
-                fused_chunk<T>(wl, c, -ref, vmax, vc, Sa, Sb, Aa, Ab);
-            }
+            FusedChunk<T, kF>::run(w, c, nrh, floor2, vmax, vc, Sa, Sb, Aa, Ab);
+        }
+        a += STEP; c += G;
+        int k = 1;
+#pragma unroll 1
+        for (; k + 4 <= KT; k += 4) {           // interior chunks, four in flight
+            const uint4 w0 = lds128(a), w1 = lds128(a + STEP), w2 = lds128(a + 2 * STEP),
+                        w3 = lds128(a + 3 * STEP);
+            FusedChunk<T, kF>::run(w0, c, nrh, floor2, vmax, vc, Sa, Sb, Aa, Ab);
+            FusedChunk<T, kF>::run(w1, c + G, nrh, floor2, vmax, vc, Sa, Sb, Aa, Ab);
+            FusedChunk<T, kF>::run(w2, c + 2 * G, nrh, floor2, vmax, vc, Sa, Sb, Aa, Ab);
+            FusedChunk<T, kF>::run(w3, c + 3 * G, nrh, floor2, vmax, vc, Sa, Sb, Aa, Ab);
+            a += 4 * STEP; c += 4 * G;
+        }
+#pragma unroll 1
+        for (; k < KT; ++k) {
+            const uint4 w = lds128(a);
+            FusedChunk<T, kF>::run(w, c, nrh, floor2, vmax, vc, Sa, Sb, Aa, Ab);
+            a += STEP; c += G;
+        }
+#pragma unroll 1
+        for (; k < ITER; ++k) {                  // may hold the row's last chunk, or lie past it
+            const int hi = c < cl ? EPC : (c == cl ? r.e_hi : 0);
+            const uint4 w = lds_keep<T>(a, keep_tab + (uint32_t)hi * 16);
+            FusedChunk<T, kF>::run(w, c, nrh, floor2, vmax, vc, Sa, Sb, Aa, Ab);
+            a += STEP; c += G;
         }
         const float Sl = (Sa.x + Sa.y) + (Sb.x + Sb.y), Al = (Aa.x + Aa.y) + (Ab.x + Ab.y);
-        // out of range, NaN, or a lane that saw nothing above the mask fill value
-        const bool bad = !(Sl < 1.0e30f) || Al != Al || (vc >= 0 && !(vmax > -1.0e29f));
+        // out of range, NaN, or a lane whose own elements are all below the fill value
+        // (with the FMA-pipe exponential also: a logit 2^120 above the reference, which that
+        // exponential does not represent, or a reference too large for the bf16 floor)
+        const bool bad = valid && has && (!(Sl < 1.0e30f) || Al != Al || !(vmax > -1.0e29f) ||
+                                          (kF && (coarse || !(fmaf(vmax, kLog2e, nrh) < 120.f))));
         RowOut out;
         if (__any_sync(0xffffffffu, bad)) {
             out = reduce_row_exact<T, G>(stage_addr, r, sub);
         } else {
-            const float m = group_max<G>(vmax);
+            const float m = group_max<G>(has ? vmax : -INFINITY);
             int cand = INT_MAX;
-            if (vc >= 0 && vmax == m) {
-                uint4 w = lds128(stage_addr + (uint32_t)vc * 16);
-                if (vc == cf || vc == cl)
-                    mask_chunk<T, true>(w, vc == cf ? r.e_lo : 0, vc == cl ? r.e_hi : EPC);
+            if (has && vmax == m) {
+                const int lo = vc == cf ? r.e_lo : 0;
+                const int hi = vc == cl ? r.e_hi : EPC;
+                const uint4 w = lds_keep<T>(stage_addr + (uint32_t)vc * 16,
+                                            keep_tab + (uint32_t)(lo * (EPC + 1) + hi) * 16);
                 float x[EPC];
                 chunk_unpack<T>(w, x);
                 int j = EPC - 1;
 #pragma unroll
-                for (int k = EPC - 2; k >= 0; --k) if (x[k] == m) j = k;
+                for (int q = EPC - 2; q >= 0; --q) if (x[q] == m) j = q;
                 cand = (vc - cf) * EPC + j - r.e_lo;
             }
             out.arg = group_min<G>(cand);
             if (out.arg == INT_MAX) out.arg = 0;
             const float mh = m * kLog2e;
             const float ml = fmaf(m, kLog2e, -mh);
-            const float d = ref - mh;                    // <= 0; lanes without chunks have S = 0
-            const float sc = ex2(d);
+            const float d = -nrh - mh;                   // <= 0 for a lane that holds chunks
+            const float sc = has ? ex2(d) : 0.f;         // a lane without chunks adds nothing
             const float S = group_sum<G>(Sl * sc);
             const float A2 = group_sum<G>(fmaf(d, Sl, Al) * sc);
             // fast logarithm and division: absolute error near 1e-6, far inside the tolerance
@@ -300,102 +431,196 @@ __device__ __forceinline__ void reduce_tile(const CtcParams &p, uint32_t stage_a
         }
         if (p.frame_logprob && valid) {
             float *o = p.frame_logprob + (r0 + i) * p.ld;
-            for (int a = sub; a < p.V; a += G)
-                o[a] = Elem<T>::load_shared(stage_addr + off + a * ES) - out.lse;
+            for (int e = sub; e < p.V; e += G)
+                o[e] = Elem<T>::load_shared(stage_addr + off + e * ES) - out.lse;
         }
     }
 }
 
-template <typename T, int G>
+struct MaxAt {
+    float v;
+    int at;
+};
+__device__ __forceinline__ MaxAt better(MaxAt a, MaxAt b) {
+    // larger value wins; on equal values the earlier frame; "at < 0" means empty
+    if (b.at >= 0 && (a.at < 0 || b.v > a.v || (b.v == a.v && b.at < a.at))) return b;
+    return a;
+}
+__device__ __forceinline__ MaxAt warp_max_at(MaxAt x) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        MaxAt y;
+        y.v = __shfl_xor_sync(0xffffffffu, x.v, o);
+        y.at = __shfl_xor_sync(0xffffffffu, x.at, o);
+        x = better(x, y);
+    }
+    return x;
+}
+
+// Adds k to a {epoch : 32 | count : 32} word and returns the count before the add.  A word
+// whose epoch is not this call's is a leftover (of an earlier call, or never written) and counts
+// as {epoch, 0}.  Epochs grow from call to call, so one atomic max with {epoch, 0} replaces a
+// leftover of an earlier call and leaves a word of this call alone; the add follows it without
+// waiting.  Only a leftover with a larger epoch field (memory that held something else) takes
+// the slow way: whoever sees it swaps {epoch, 0} in, and nobody adds before that has happened.
+__device__ __forceinline__ uint32_t tagged_finish(unsigned long long *w, uint32_t epoch, uint32_t k,
+                                                  unsigned long long old, bool &ok) {
+    if ((uint32_t)(old >> 32) == epoch) return (uint32_t)old;
+    const unsigned long long tag = (unsigned long long)epoch << 32;
+    for (int tries = 0; tries < (1 << 16); ++tries) {
+        const unsigned long long cur = *reinterpret_cast<volatile unsigned long long *>(w);
+        if ((uint32_t)(cur >> 32) == epoch) return (uint32_t)atomicAdd(w, (unsigned long long)k);
+        atomicCAS(w, cur, tag);
+    }
+    ok = false;
+    return 0xffffffffu;
+}
+__device__ __forceinline__ unsigned long long tagged_begin(unsigned long long *w, uint32_t epoch,
+                                                           uint32_t k) {
+    atomicMax(w, (unsigned long long)epoch << 32);
+    return atomicAdd(w, (unsigned long long)k);
+}
+// Shared memory: one mbarrier per warp | keep table | the warps' stages.
+//
+// Tiles: a warp's first tile is tile number (its index among all warps); further tiles are
+// claimed one at a time from counters in the workspace, so that SMs that run ahead take more and
+// all finish together.  One counter could not keep up (atomics on one address retire about 190
+// per microsecond; tiles of 16 KB are finished at twice that rate), so there are C of them, C
+// the largest of 4, 3, 2, 1 that divides the warps per CTA: counter c hands out the tiles GW +
+// c, GW + c + C, ... and serves warps c, c + C, ... of every CTA, so that all counters have the
+// same number of tiles and of warps and run out together.  The claim for the tile after the
+// current one is in flight while the current one is worked on.
+template <typename T, int G, int kF>
 __global__ void __launch_bounds__(768, 1) ctc_rows_tma(const CtcParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
-    constexpr int ES = Elem<T>::kBytes;
+    constexpr int ES = Elem<T>::kBytes, EPC = Elem<T>::kPerChunk;
     pdl_launch_dependents();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int W = p.warps, S = p.stages, R = p.rows_per_tile;
-    // Tile j goes to CTA j mod grid, and within the CTA to warp (j / grid) mod W: every CTA
-    // gets the same number of tiles (give or take one) whatever the size of the matrix.
+    const int W = p.warps, R = p.rows_per_tile;
     const int64_t gw = (int64_t)blockIdx.x + (int64_t)gridDim.x * warp, GW = (int64_t)gridDim.x * W;
-    const int64_t my_tiles = gw < p.num_tiles ? (p.num_tiles - gw + GW - 1) / GW : 0;
-    if (my_tiles == 0) return;
 
-    const uint32_t bar0 = smem_u32(smem) + (warp * S) * 8;
-    const uint32_t stage_region = (uint32_t)((W * S * 8 + 127) & ~127);
-    const uint32_t stage0 = smem_u32(smem) + stage_region + (uint32_t)(warp * S) * p.stage_stride;
-    unsigned char *stage0_ptr = smem + stage_region + (size_t)(warp * S) * p.stage_stride;
+    const uint32_t bar = smem_u32(smem) + warp * 8;
+    const uint32_t tab_off = (uint32_t)((W * 8 + 15) & ~15);
+    const uint32_t keep_tab = smem_u32(smem) + tab_off;
+    const uint32_t stage_region = (tab_off + (uint32_t)(EPC * (EPC + 1)) * 16 + 127) & ~127u;
+    const uint32_t stage = smem_u32(smem) + stage_region + (uint32_t)warp * p.stage_stride;
+    unsigned char *stage_ptr = smem + stage_region + (size_t)warp * p.stage_stride;
 
+    build_keep_table<T>(reinterpret_cast<uint4 *>(smem + tab_off), (int)threadIdx.x, (int)blockDim.x);
     if (lane == 0) {
-        for (int s = 0; s < S; ++s) mbar_init(bar0 + s * 8, 1);
+        mbar_init(bar, 1);
         mbar_init_fence();
     }
-    __syncwarp();
+    __syncthreads();                       // the keep table is shared by all warps
+    if (gw >= p.num_tiles) return;
 
     const uintptr_t base = reinterpret_cast<uintptr_t>(p.logits);
     const int64_t row_pitch = p.ld * ES;
 
-    // Brings tile k of this warp into stage s.  The tile's rows are one contiguous byte range
+    // Brings tile t into this warp's stage.  The tile's rows are one contiguous byte range
     // (padding between rows included); the 16-byte-aligned superset of the range is fetched with
     // one bulk copy, except where that superset would leave the matrix (near its two ends):
     // there the copy is one chunk shorter and the few elements outside it are fetched with
     // plain loads.  Bytes of neighbouring rows that come along are never looked at.
-    auto issue = [&](int64_t k, int s) {
-        const ranges::TileReads t = ranges::tile_reads(base, p.total_bytes, row_pitch,
-                                                       (int64_t)p.V * ES, p.N, R, gw + k * GW);
-        const uint32_t bar = bar0 + s * 8;
-        unsigned char *dst = stage0_ptr + (size_t)s * p.stage_stride;
-        if (t.head_hi > t.head_lo || t.tail_hi > t.tail_lo) {
+    auto issue = [&](int64_t t) {
+        const ranges::TileReads tr = ranges::tile_reads(base, p.total_bytes, row_pitch,
+                                                        (int64_t)p.V * ES, p.N, R, t);
+        if (tr.head_hi > tr.head_lo || tr.tail_hi > tr.tail_lo) {
             for (int side = 0; side < 2; ++side) {
-                const uintptr_t lo = side ? t.tail_lo : t.head_lo, hi = side ? t.tail_hi : t.head_hi;
+                const uintptr_t lo = side ? tr.tail_lo : tr.head_lo, hi = side ? tr.tail_hi : tr.head_hi;
                 for (uintptr_t a = lo + (uintptr_t)lane * ES; a < hi; a += 32 * ES) {
-                    if (ES == 4) *reinterpret_cast<uint32_t *>(dst + (a - t.f0)) =
+                    if (ES == 4) *reinterpret_cast<uint32_t *>(stage_ptr + (a - tr.f0)) =
                             *reinterpret_cast<const uint32_t *>(a);
-                    else *reinterpret_cast<uint16_t *>(dst + (a - t.f0)) =
+                    else *reinterpret_cast<uint16_t *>(stage_ptr + (a - tr.f0)) =
                             *reinterpret_cast<const uint16_t *>(a);
                 }
             }
             __syncwarp();
         }
         if (lane == 0) {
-            if (t.bulk_hi > t.bulk_lo) {
-                const uint32_t bytes = (uint32_t)(t.bulk_hi - t.bulk_lo);
+            if (tr.bulk_hi > tr.bulk_lo) {
+                const uint32_t bytes = (uint32_t)(tr.bulk_hi - tr.bulk_lo);
                 fence_proxy_async();
                 mbar_arrive_expect_tx(bar, bytes);
-                bulk_g2s(stage0 + (uint32_t)s * p.stage_stride + (uint32_t)(t.bulk_lo - t.f0),
-                         reinterpret_cast<const void *>(t.bulk_lo), bytes, bar);
+                bulk_g2s(stage + (uint32_t)(tr.bulk_lo - tr.f0),
+                         reinterpret_cast<const void *>(tr.bulk_lo), bytes, bar);
             } else {
                 mbar_arrive(bar);
             }
         }
     };
 
-    pdl_wait();
-    const int prologue = (int)min((int64_t)S, my_tiles);
-    for (int k = 0; k < prologue; ++k) issue(k, k);
-
-    bool failed = false;
-    int s = 0;
+    const bool dynamic = p.tile_counter != nullptr && p.num_tiles > GW;
+    const int C = p.counters;
+    unsigned long long *counter = p.tile_counter + (warp % C) * 32;
+    const int64_t first = GW + warp % C;                 // tile of this counter's slot 0
+    bool failed = false, ok = true;
     uint32_t parity = 0;
-    int64_t k = 0;
-    for (; k < my_tiles; ++k) {
-        if (!mbar_wait_bounded(bar0 + s * 8, parity)) { failed = true; break; }
-        const int64_t r0 = (gw + k * GW) * R;
+    // this warp's tiles: t, t + step, ... up to (not including) t_end
+    int64_t t = gw, t_end = gw + 1, step = 1;
+    unsigned long long pend = 0;          // lane 0: the counter word before the claim in flight
+    uint32_t pend_k = 0;
+    auto claim_begin = [&]() {
+        pend_k = p.claim;
+        if (lane == 0) pend = tagged_begin(counter, p.epoch, pend_k);
+    };
+    pdl_wait();
+    issue(t);
+    if (dynamic) claim_begin();
+    while (t < p.num_tiles) {
+        if (!mbar_wait_bounded(bar, parity)) { failed = true; break; }
+        parity ^= 1u;
+        const int64_t r0 = t * R;
         const int nrows = (int)min((int64_t)R, p.N - r0);
         const uint32_t head = (uint32_t)((base + (uintptr_t)(r0 * row_pitch)) & 15);
-        reduce_tile<T, G>(p, stage0 + (uint32_t)s * p.stage_stride, head, r0, nrows, lane);
+        reduce_tile<T, G, kF>(p, stage, keep_tab, head, r0, nrows, lane);
         __syncwarp();
-        if (k + S < my_tiles) issue(k + S, s);
-        if (++s == S) { s = 0; parity ^= 1u; }
+        int64_t nt = dynamic ? t + step : t + GW;
+        if (dynamic && nt >= t_end) {
+            // the claimed tiles are used up: take the claim in flight, start the next one
+            uint32_t cnt = 0;
+            if (lane == 0) cnt = tagged_finish(counter, p.epoch, pend_k, pend, ok);
+            cnt = __shfl_sync(0xffffffffu, cnt, 0);
+            if (!__shfl_sync(0xffffffffu, (int)ok, 0)) { failed = true; break; }
+            step = C;
+            nt = first + (int64_t)cnt * C;
+            t_end = nt + (int64_t)pend_k * C;
+            if (nt < p.num_tiles) claim_begin();
+        }
+        if (nt < p.num_tiles) issue(nt);
+        t = nt;
     }
     if (failed) {
-        // A wait ran out: poison every frame this warp still owed so that the per-utterance
+        // A wait ran out, or the tile counter could not be read: poison the frames of the tiles
+        // this warp still holds and of one more, unclaimed one, so that the per-utterance
         // kernel reports SSD_UTT_INTERNAL, then let copies that may be in flight land.
-        for (; k < my_tiles; ++k) {
-            const int64_t r0 = (gw + k * GW) * R;
+        for (; t < p.num_tiles && (!dynamic || t < t_end); t += dynamic ? step : GW) {
+            const int64_t r0 = t * R;
             const int nrows = (int)min((int64_t)R, p.N - r0);
             for (int i = lane; i < nrows; i += 32) {
                 p.frame_entropy[r0 + i] = __uint_as_float(kNanInternal);
                 p.frame_argmax[r0 + i] = 0;
                 if (p.frame_lse) p.frame_lse[r0 + i] = __uint_as_float(kNanInternal);
+            }
+        }
+        if (dynamic) {
+            // the claim in flight: its tiles are this warp's as well
+            uint32_t cnt = 0xffffffffu;
+            if (lane == 0 && (uint32_t)(pend >> 32) == p.epoch) cnt = (uint32_t)pend;
+            cnt = __shfl_sync(0xffffffffu, cnt, 0);
+            if (cnt != 0xffffffffu) {
+                t = first + (int64_t)cnt * C;
+                for (t_end = t + (int64_t)pend_k * C; t < p.num_tiles && t < t_end; t += C) {
+                    const int64_t r0 = t * R;
+                    const int nrows = (int)min((int64_t)R, p.N - r0);
+                    for (int i = lane; i < nrows; i += 32) {
+                        p.frame_entropy[r0 + i] = __uint_as_float(kNanInternal);
+                        p.frame_argmax[r0 + i] = 0;
+                        if (p.frame_lse) p.frame_lse[r0 + i] = __uint_as_float(kNanInternal);
+                    }
+                }
+            } else if (lane == 0) {
+                p.frame_entropy[0] = __uint_as_float(kNanInternal);   // the counter itself failed
             }
         }
         drain_after_error();
@@ -450,25 +675,6 @@ __global__ void __launch_bounds__(256) ctc_rows_plain(const CtcParams p) {
 // of up to 1024 frames in one sweep, and the loads of a sweep are issued together.
 constexpr int kUttThreads = 1024;
 
-struct MaxAt {
-    float v;
-    int at;
-};
-__device__ __forceinline__ MaxAt better(MaxAt a, MaxAt b) {
-    // larger value wins; on equal values the earlier frame; "at < 0" means empty
-    if (b.at >= 0 && (a.at < 0 || b.v > a.v || (b.v == a.v && b.at < a.at))) return b;
-    return a;
-}
-__device__ __forceinline__ MaxAt warp_max_at(MaxAt x) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        MaxAt y;
-        y.v = __shfl_xor_sync(0xffffffffu, x.v, o);
-        y.at = __shfl_xor_sync(0xffffffffu, x.at, o);
-        x = better(x, y);
-    }
-    return x;
-}
 // Maximum over the block; valid in warp 0 (all its lanes).  One __syncthreads.
 __device__ __forceinline__ MaxAt block_max_at(MaxAt x, MaxAt *scratch /* [32] shared */) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
@@ -603,6 +809,22 @@ __global__ void __launch_bounds__(kUttThreads) gate_kernel(
     }
 }
 
+// Eq. 3 from per-utterance maxima that ssd_ctc_draft left behind: utterance b passes iff its
+// largest frame entropy is below tau and no frame was NaN (status bits), its offsets were sound
+// and no wait ran out.  An utterance without frames has maximum 0.
+__global__ void __launch_bounds__(256) gate_from_maxima_kernel(
+    const float *__restrict__ utt_max_entropy, const uint32_t *__restrict__ utt_status, int B,
+    float tau, uint8_t *__restrict__ gate_accept, float *__restrict__ max_entropy) {
+    pdl_enter();
+    for (int b = blockIdx.x * blockDim.x + threadIdx.x; b < B; b += gridDim.x * blockDim.x) {
+        const float h = utt_max_entropy[b];
+        const uint32_t st = utt_status[b];
+        const bool sound = (st & (SSD_UTT_NONFINITE | SSD_UTT_BAD_OFFSETS | SSD_UTT_INTERNAL)) == 0;
+        gate_accept[b] = (sound && h < tau) ? 1 : 0;
+        max_entropy[b] = h;
+    }
+}
+
 int g_sm_count = 0;
 int sm_count() {
     if (g_sm_count == 0) {
@@ -626,26 +848,37 @@ unsigned long long next_epoch() {
 }
 
 // Kernel and launch shape of the frame-statistics pass for these sizes.
-// G lanes share a row (so that a lane walks about 8..18 chunks of 16 bytes), a warp works on
-// 32/G rows at a time, and a tile is a whole number of such row groups of about 8 KB.
-int plan_ctc(ssd_dtype dtype, int V, int64_t ld, int64_t N, const ssd_launch_opts *o, CtcPlan *plan) {
+// G lanes share a row, a warp works on 32/G rows at a time (one pass), and a tile is a whole
+// number of passes.  Few lanes per row spread the per-pass work (row geometry, masked first and
+// last iterations, lane merges, logarithms, stores) over more rows; one pass of about 16 KB per
+// warp and as many warps as shared memory holds keep both the copies and the arithmetic busy.
+int plan_ctc(ssd_dtype dtype, int V, int64_t ld, int64_t N, int B, const ssd_launch_opts *o,
+             CtcPlan *plan) {
     const int es = dtype == SSD_F32 ? 4 : 2;
     CtcPlan pl{};
     int kernel = o ? o->kernel : 0;
     const int64_t row_pitch = ld * es;
     const int64_t row_bytes = (int64_t)V * es;
-    const int64_t chunks = (row_bytes + 15) / 16 + 1;
-    const int G = chunks <= 72 ? 4 : chunks <= 144 ? 8 : chunks <= 288 ? 16 : 32;
+    const int64_t chunks_max = (row_bytes + 31 - es) / 16;   // most 16-byte chunks a row touches
+    const int64_t chunks_min = (row_bytes + 15) / 16;
+    // lanes per row: the smallest power of two for which one pass (32/G rows) is at most 16.5 KB
+    int G = 2;
+    while (G < 32 && (32 / G) * row_pitch > 16896) G *= 2;
+    if (o && o->split > 0) {
+        G = o->split;
+        if (G != 2 && G != 4 && G != 8 && G != 16 && G != 32) return SSD_ERR_ARG;
+    }
     const int rpw = 32 / G;
-    const int smem_budget = 200 * 1024;
-    // One stage per warp and as many warps as fit hide the copy latency behind other warps'
-    // arithmetic and give the schedulers more independent work than a deeper ring with fewer
-    // warps does; a small matrix (a tile or two per warp) is better off prefetching.
-    const int64_t tiles_guess = N * row_pitch / 8192 + 1;
+    const int iters = (int)((chunks_max + G - 1) / G);
+    // a forced G that makes a lane add up thousands of terms by itself costs accuracy: refused
+    if (o && o->split > 0 && iters > 160 && G < 32) return SSD_ERR_ARG;
+    int tail_from = (int)((chunks_min - 1) / G);
+    if (tail_from < 1) tail_from = 1;
+    (void)B;
+    const int epc = 16 / es;
+    const int64_t fixed = 24 * 8 + 16 + (int64_t)epc * (epc + 1) * 16 + 128;
+    const int64_t stage_budget = 216 * 1024 - fixed;
     int warps = 0, R = 0;
-    int stages = (o && o->stages > 0) ? o->stages : (tiles_guess < 2ll * 24 * sm_count() ? 2 : 1);
-    if (stages < 1) stages = 1;
-    if (stages > 8) stages = 8;
     int64_t stage_stride = 0;
     if (kernel != 1 && row_pitch <= 2 * row_bytes + 64 && row_pitch < (1 << 20)) {
         int64_t groups = 8192 / (rpw * row_pitch);
@@ -653,31 +886,49 @@ int plan_ctc(ssd_dtype dtype, int V, int64_t ld, int64_t N, const ssd_launch_opt
         if (o && o->stage_bytes > 0) groups = (o->stage_bytes + rpw - 1) / rpw;
         for (; groups >= 1 && warps == 0; groups = groups > 1 ? groups / 2 : 0) {
             R = (int)(groups * rpw);
-            stage_stride = ((R - 1) * row_pitch + row_bytes + 32 + 127) & ~127ll;
-            int64_t w = (smem_budget - 1024) / (stages * stage_stride);
+            // the last row's lanes read iters * G chunks from the row's first chunk on, whether
+            // the row reaches that far or not (what lies past it is masked, not used)
+            stage_stride = ((R - 1) * row_pitch + 16 + (int64_t)iters * G * 16 + 127) & ~127ll;
+            int64_t w = stage_budget / stage_stride;
             if (w > 24) w = 24;
+            if (w >= 5 && w % 2 && w % 3) --w;      // so that 2 or more tile counters divide it
             if (o && o->warps > 0 && o->warps < w) w = o->warps;
             if (w >= 1) warps = (int)w;
         }
     }
     if (warps == 0) {
-        if (kernel == 2) return SSD_ERR_ARG;   // forced, but a row group does not fit a stage
+        if (kernel == 2) return SSD_ERR_ARG;   // forced, but a pass does not fit a stage
         kernel = 1;
     } else {
         kernel = 2;
     }
     pl.kernel = kernel; pl.lanes_per_row = G; pl.rows_per_tile = R; pl.warps = warps;
-    pl.stages = stages; pl.stage_stride = (int)stage_stride;
-    pl.num_tiles = kernel == 2 ? (N + R - 1) / R : 0;
+    pl.stages = 1; pl.stage_stride = (int)stage_stride;
+    pl.iters = iters; pl.tail_from = tail_from;
+    pl.fma_exp = (o && o->fma_exp > 0 && dtype == SSD_BF16) ? (o->fma_exp > 2 ? 2 : o->fma_exp) : 0;
+    pl.num_tiles = kernel != 1 ? (N + R - 1) / R : 0;
+    pl.smem_bytes = kernel != 1
+        ? (size_t)(((((warps * 8 + 15) & ~15) + epc * (epc + 1) * 16) + 127) & ~127) +
+          (size_t)warps * stage_stride
+        : 0;
+    pl.workspace_bytes = 2048;      // the tile counters, 256 bytes apart, and room to spare
     *plan = pl;
     return SSD_OK;
 }
 
+namespace {
+template <typename T, int kF> void (*pick_ctc(int G))(const CtcParams) {
+    return G == 2 ? ctc_rows_tma<T, 2, kF> : G == 4 ? ctc_rows_tma<T, 4, kF>
+         : G == 8 ? ctc_rows_tma<T, 8, kF> : G == 16 ? ctc_rows_tma<T, 16, kF>
+                                                     : ctc_rows_tma<T, 32, kF>;
+}
+}  // namespace
+
+// Frame statistics of all N rows.  workspace: 256 bytes for the tile counter, or NULL (tiles are
+// then dealt out in a fixed order).
 int launch_ctc_rows(const void *logits, ssd_dtype dtype, int V, int64_t ld, int64_t N,
-                    const int64_t *frame_off, int B, float *frame_entropy, int32_t *frame_argmax,
-                    float *frame_lse, float *frame_logprob, uint32_t *utt_status,
-                    const Launch &L) {
-    (void)frame_off; (void)B; (void)utt_status;
+                    float *frame_entropy, int32_t *frame_argmax, float *frame_lse,
+                    float *frame_logprob, void *workspace, const CtcPlan &plan, const Launch &L) {
     if (N == 0) return SSD_OK;
     const ssd_launch_opts *o = L.opts;
     const int es = dtype == SSD_F32 ? 4 : 2;
@@ -687,36 +938,34 @@ int launch_ctc_rows(const void *logits, ssd_dtype dtype, int V, int64_t ld, int6
     p.total_bytes = (N - 1) * ld * es + (int64_t)V * es;
     p.frame_entropy = frame_entropy; p.frame_argmax = frame_argmax; p.frame_lse = frame_lse;
     p.frame_logprob = frame_logprob;
-    CtcPlan plan;
-    const int prc = plan_ctc(dtype, V, ld, N, o, &plan);
-    if (prc != SSD_OK) return prc;
     const int kernel = plan.kernel, G = plan.lanes_per_row, R = plan.rows_per_tile;
-    const int warps = plan.warps, stages = plan.stages;
-    const int64_t stage_stride = plan.stage_stride;
     cudaError_t e;
     if (o && o->ev_begin) {
         e = cudaEventRecord(static_cast<cudaEvent_t>(o->ev_begin), L.stream);
         if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
     }
-    if (kernel == 2) {
-        p.rows_per_tile = R; p.stages = stages; p.warps = warps;
-        p.stage_stride = (int)stage_stride;
+    if (kernel != 1) {
+        p.rows_per_tile = R; p.stages = 1; p.warps = plan.warps;
+        p.stage_stride = plan.stage_stride;
+        p.iters = plan.iters; p.tail_from = plan.tail_from;
         p.num_tiles = (N + R - 1) / R;
-        const size_t smem = (size_t)((warps * stages * 8 + 127) & ~127) +
-                            (size_t)warps * stages * p.stage_stride;
-        int64_t ctas = p.num_tiles;
+        p.tile_counter = static_cast<unsigned long long *>(workspace);
+        p.epoch = (uint32_t)next_epoch();
+        p.counters = plan.warps % 4 == 0 ? 4 : plan.warps % 3 == 0 ? 3 : plan.warps % 2 == 0 ? 2 : 1;
+        // small tiles are finished faster than a counter hands them out one by one
+        p.claim = (int64_t)R * ld * es * p.counters < 3 * 12288 ? 2 : 1;
+        int64_t ctas = (p.num_tiles + plan.warps - 1) / plan.warps;
         const int max_ctas = (o && o->ctas > 0) ? o->ctas : sm_count();
         if (ctas > max_ctas) ctas = max_ctas;
         void (*kern)(const CtcParams) = nullptr;
-        if (dtype == SSD_F32)
-            kern = G == 4 ? ctc_rows_tma<float, 4> : G == 8 ? ctc_rows_tma<float, 8>
-                 : G == 16 ? ctc_rows_tma<float, 16> : ctc_rows_tma<float, 32>;
-        else
-            kern = G == 4 ? ctc_rows_tma<bf16_t, 4> : G == 8 ? ctc_rows_tma<bf16_t, 8>
-                 : G == 16 ? ctc_rows_tma<bf16_t, 16> : ctc_rows_tma<bf16_t, 32>;
-        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (dtype == SSD_F32) kern = pick_ctc<float, 0>(G);
+        else kern = plan.fma_exp == 2 ? pick_ctc<bf16_t, 2>(G)
+                  : plan.fma_exp == 1 ? pick_ctc<bf16_t, 1>(G) : pick_ctc<bf16_t, 0>(G);
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)plan.smem_bytes);
         if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
-        e = launch_pdl(kern, (unsigned)ctas, (unsigned)(warps * 32), smem, L.stream, p);
+        e = launch_pdl(kern, (unsigned)ctas, (unsigned)(plan.warps * 32), plan.smem_bytes,
+                       L.stream, p);
         if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
     } else {
         int64_t ctas = (N + 7) / 8;
@@ -744,6 +993,18 @@ int launch_collapse(const int32_t *frame_argmax, const float *frame_entropy,
     cudaError_t e = launch_pdl(collapse_kernel, (unsigned)B, (unsigned)kUttThreads, 0, stream,
         frame_argmax, frame_entropy, frame_off, B, N, blank_id, max_draft_len, draft_tokens,
         draft_frames, draft_len, draft_full_len, utt_max_entropy, utt_status);
+    if (e == cudaSuccess) e = cudaGetLastError();
+    if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
+    return SSD_OK;
+}
+
+int launch_gate_from_maxima(const float *utt_max_entropy, const uint32_t *utt_status, int B,
+                            float tau, uint8_t *gate_accept, float *max_entropy,
+                            cudaStream_t stream) {
+    if (B == 0) return SSD_OK;
+    const unsigned grid = (unsigned)((B + 255) / 256 < 8 ? (B + 255) / 256 : 8);
+    cudaError_t e = launch_pdl(gate_from_maxima_kernel, grid, 256u, 0, stream, utt_max_entropy,
+                               utt_status, B, tau, gate_accept, max_entropy);
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
     return SSD_OK;

@@ -31,7 +31,7 @@ int32_t ssd_ctc_draft_read_span(uint64_t base_addr, ssd_dtype dtype, int32_t V, 
     const int es = dtype == SSD_F32 ? 4 : 2;
     if (base_addr % es) return SSD_ERR_ALIGN;
     CtcPlan plan;
-    const int rc = plan_ctc(dtype, V, ld, N, opts, &plan);
+    const int rc = plan_ctc(dtype, V, ld, N, 0, opts, &plan);
     if (rc != SSD_OK) return rc;
     const int64_t row_pitch = ld * es, row_bytes = (int64_t)V * es;
     const int64_t total = N > 0 ? (N - 1) * row_pitch + row_bytes : 0;

@@ -79,6 +79,16 @@ def compare_stage1(gpu, gate, orc, frame_off, tau_ctc, require_all_margins=True)
                 max_dlse=float(dL.max()) if dL.size else 0.0)
 
 
+def check_gate_from_maxima(ctc_out, gate, tau_ctc):
+    """ssd_entropy_gate's second form (from ssd_ctc_draft's utterance maxima and status words)
+    against its first form (from the frame entropies): the same decisions and maxima, bit for
+    bit; the first form is what compare_stage1 holds against the oracle."""
+    g2 = ssd.ssd_entropy_gate_from_maxima(ctc_out["utt_max_entropy"], ctc_out["utt_status"], tau_ctc)
+    torch.cuda.synchronize()
+    assert torch.equal(g2["gate_accept"], gate["gate_accept"])
+    assert torch.equal(g2["max_entropy"].view(torch.int32), gate["max_entropy"].view(torch.int32))
+
+
 def compare_stage2(gpu, orc, tok_off, tau_slm, skip=None, require_all_margins=True):
     off = np.asarray(tok_off)
     B = len(off) - 1
@@ -146,6 +156,9 @@ def guarded_ctc_outputs(N, B, device):
                draft_frames=g.alloc(N, torch.int32), draft_len=g.alloc(B, torch.int32),
                draft_full_len=g.alloc(B, torch.int32), utt_max_entropy=g.alloc(B, torch.float32),
                utt_status=g.alloc(B, torch.int32))
+    ws = g.alloc(64 + 512, torch.int32)                      # 256-byte aligned slice of it
+    shift = ((-ws.data_ptr()) % 256) // 4
+    out["workspace"] = ws[shift:shift + 512].view(torch.uint8)
     return g, out
 
 

@@ -38,11 +38,13 @@ def test_status_strings(lib):
     assert lib.ssd_version() >= 100
 
 
-def _ctc(lib, logits=8, dtype=1, V=10, ld=10, off=8, B=1, N=4, blank=0, cap=5, outs=8):
+def _ctc(lib, logits=8, dtype=1, V=10, ld=10, off=8, B=1, N=4, blank=0, cap=5, outs=8, ws=0,
+         ws_bytes=0):
     p = C.c_void_p
     o = p(outs) if outs else None
     return lib.ssd_ctc_draft(p(logits) if logits else None, dtype, V, ld, p(off) if off else None,
-                             B, N, blank, cap, o, o, o, None, o, o, o, o, o, o, None, 0, None, None)
+                             B, N, blank, cap, o, o, o, None, o, o, o, o, o, o,
+                             p(ws) if ws else None, ws_bytes, None, None)
 
 
 def test_ctc_draft_rejects_bad_arguments_on_the_host(lib):
@@ -59,6 +61,8 @@ def test_ctc_draft_rejects_bad_arguments_on_the_host(lib):
     assert _ctc(lib, outs=0) == ssd.ERR_NULL
     assert _ctc(lib, logits=9, dtype=1) == ssd.ERR_ALIGN     # bf16 at an odd address
     assert _ctc(lib, logits=10, dtype=0) == ssd.ERR_ALIGN    # fp32 at 2 mod 4
+    assert _ctc(lib, ws=256, ws_bytes=2047) == ssd.ERR_WORKSPACE     # 2048 bytes needed
+    assert _ctc(lib, ws=264, ws_bytes=4096) == ssd.ERR_WORKSPACE     # not 256-byte aligned
 
 
 def _verify(lib, logits=8, dtype=1, V=10, ld=10, off=8, ids=8, B=1, M=4, outs=8, ws=256, ws_bytes=1 << 20):
@@ -100,14 +104,18 @@ def test_verify_rejects_bad_options(lib):
 
 def test_gate_rejects_bad_arguments_on_the_host(lib):
     p = C.c_void_p
-    assert lib.ssd_entropy_gate(p(8), p(8), -1, 4, C.c_float(0.5), p(8), p(8), None, None) == ssd.ERR_ARG
-    assert lib.ssd_entropy_gate(None, p(8), 1, 4, C.c_float(0.5), p(8), p(8), None, None) == ssd.ERR_NULL
-    assert lib.ssd_entropy_gate(p(8), None, 1, 4, C.c_float(0.5), p(8), p(8), None, None) == ssd.ERR_NULL
-    assert lib.ssd_entropy_gate(p(8), p(8), 1, 4, C.c_float(0.5), None, p(8), None, None) == ssd.ERR_NULL
+    g = lambda *a: lib.ssd_entropy_gate(*a)
+    assert g(p(8), p(8), -1, 4, C.c_float(0.5), p(8), p(8), None, None, None, None) == ssd.ERR_ARG
+    assert g(None, p(8), 1, 4, C.c_float(0.5), p(8), p(8), None, None, None, None) == ssd.ERR_NULL
+    assert g(p(8), None, 1, 4, C.c_float(0.5), p(8), p(8), None, None, None, None) == ssd.ERR_NULL
+    assert g(p(8), p(8), 1, 4, C.c_float(0.5), None, p(8), None, None, None, None) == ssd.ERR_NULL
+    # the form that reads utterance maxima needs their status words as well
+    assert g(None, None, 1, 0, C.c_float(0.5), p(8), p(8), None, p(8), None, None) == ssd.ERR_NULL
+    assert g(None, None, 1, 0, C.c_float(0.5), None, p(8), None, p(8), p(8), None) == ssd.ERR_NULL
 
 
 def test_workspace_queries(lib):
-    assert ssd.ssd_ctc_draft_workspace_bytes(32, 16000, 1025, ssd.BF16) == 0
+    assert ssd.ssd_ctc_draft_workspace_bytes(32, 16000, 1025, ssd.BF16) == 2048
     small = ssd.ssd_verify_workspace_bytes(1, 250, 152064, ssd.BF16)
     big = ssd.ssd_verify_workspace_bytes(32, 6400, 49152, ssd.BF16)
     assert small >= 256 + 250 * 8 * 8 and big >= 256 + 6400 * 8 * 8

@@ -50,6 +50,7 @@ def test_stage1_random(cuda_device, seed):
     gate = ssd.ssd_entropy_gate(out["frame_entropy"], offd, tau)
     torch.cuda.synchronize()
     g.check()
+    H.check_gate_from_maxima(out, gate, tau)
     orc = H.oracle_stage1(H.storage_numpy(wide[:, col0:col0 + V].contiguous()), V, off, blank, cap, tau)
     H.compare_stage1(out, gate, orc, off, tau, require_all_margins=False)
 

@@ -28,6 +28,7 @@ def run_stage1(logits_dev, frame_off, V, blank_id, cap, tau, kernel, guard=True,
     torch.cuda.synchronize()
     if g:
         g.check()
+    H.check_gate_from_maxima(out, gate, tau)
     return out, gate
 
 
@@ -213,3 +214,138 @@ def test_pipeline_shapes(cuda_device, warps, stages, rows):
     """Other ring shapes of the bulk-copy kernel give the same answers."""
     w = synth.scaled(synth.CONFIGS[1], B=3, seed=21)
     check_workload(w, cuda_device, 2, warps=warps, stages=stages, stage_bytes=rows, ctas=5)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("V", [1, 5, 17, 24, 129])
+@pytest.mark.parametrize("shift", [-100.0, -200.0, 90.0])
+def test_short_rows_far_from_zero(cuda_device, dtype, V, shift):
+    """Rows with fewer 16-byte chunks than lanes share them, all logits moved by a constant
+    (Eq. 2 / Eq. 3 do not change under it): lanes that hold no chunk of a row must add nothing,
+    whatever the row maximum is."""
+    w = synth.scaled(synth.CONFIGS[1], B=4, V_ctc=V, dtype=dtype, variant="literal",
+                     tau_ctc=0.9, seed=500 + V, max_draft_len=30)
+    cb = synth.make_ctc_batch(w, "cpu", [33, 2, 0, 50])
+    x = (cb.logits.float() + shift).to(cb.logits.dtype)
+    for G in (0, 2, 4, 8, 32):
+        out, gate = run_stage1(x.to(cuda_device), cb.frame_off, V, 0, 30, 0.9, 2, split=G)
+        st = H.status_u32(out["utt_status"])
+        assert not (st & ssd.UTT_NONFINITE).any()
+        orc = H.oracle_stage1(H.storage_numpy(x), V, cb.frame_off.numpy(), 0, 30, 0.9)
+        H.compare_stage1(out, gate, orc, cb.frame_off.numpy(), 0.9, require_all_margins=False)
+
+
+@pytest.mark.parametrize("V,dtype", [(1025, "bf16"), (348, "bf16"), (4097, "bf16"), (129, "f32"),
+                                     (1025, "f32"), (2049, "bf16"), (64, "bf16"), (7, "bf16")])
+def test_lanes_per_row_and_exponential_split(cuda_device, V, dtype):
+    """Every number of lanes per row the kernel is built for, and the FMA-pipe exponential on
+    one or two of a bf16 chunk's four pairs, give the oracle's answers."""
+    w = synth.scaled(synth.CONFIGS[1], B=5, V_ctc=V, dtype=dtype, t_lo=37, t_hi=211, seed=40 + V)
+    cb = synth.make_ctc_batch(w, "cpu")
+    x = cb.logits.to(cuda_device)
+    orc = H.oracle_stage1(H.storage_numpy(cb.logits), V, cb.frame_off.numpy(), w.blank_id,
+                          w.max_draft_len, w.tau_ctc)
+    variants = [dict(split=G) for G in (2, 4, 8, 16, 32)]
+    if dtype == "bf16":
+        variants += [dict(fma_exp=1), dict(fma_exp=2), dict(split=8, fma_exp=1)]
+    ran = 0
+    for kw in variants:
+        try:
+            out, gate = run_stage1(x, cb.frame_off, V, w.blank_id, w.max_draft_len, w.tau_ctc, 0, **kw)
+        except ssd.SsdError as e:        # few lanes on a long row: refused for accuracy
+            assert e.code == ssd.ERR_ARG and kw.get("split", 32) < 32
+            continue
+        ran += 1
+        H.compare_stage1(out, gate, orc, cb.frame_off.numpy(), w.tau_ctc, require_all_margins=False)
+    assert ran >= 3
+
+
+def test_fma_exponential_range_guards(cuda_device):
+    """The FMA-pipe exponential represents neither 2^t for t above 120 nor references beyond
+    +-4096 (its lower clamp is a bf16 value): such rows must take the exact routine."""
+    V, T = 1025, 24
+    g = torch.Generator().manual_seed(8)
+    x = torch.randn((T, V), generator=g)
+    x[0:8, 700] += 200.0                 # far above the first chunk's reference
+    x[8:16] += 6000.0                    # large reference
+    x[16:24] -= 9000.0
+    x[16:24, 3] += 150.0
+    x = x.to(torch.bfloat16)
+    off = torch.tensor([0, 8, 16, 24], dtype=torch.int64)
+    orc = H.oracle_stage1(H.storage_numpy(x), V, off.numpy(), 0, T, 1.0)
+    for f in (1, 2):
+        out, gate = run_stage1(x.to(cuda_device), off, V, 0, T, 1.0, 2, fma_exp=f)
+        np.testing.assert_array_equal(out["frame_argmax"].cpu().numpy(), orc["frame_argmax"])
+        d = np.abs(out["frame_entropy"].cpu().numpy().astype(np.float64) - orc["frame_entropy"])
+        assert d.max() <= H.FLOAT_TOL
+        # lse is thousands here: one fp32 ulp at that size is beyond 1e-4 absolute
+        lse, want = out["frame_lse"].cpu().numpy().astype(np.float64), orc["frame_lse"]
+        assert (np.abs(lse - want) <= 1e-4 + 2 * np.spacing(np.abs(want).astype(np.float32))).all()
+
+
+def test_many_short_utterances_per_tile(cuda_device):
+    """Utterances of 0 to 3 frames, empty ones between them: a tile of frames spans dozens."""
+    rng = np.random.default_rng(77)
+    lens = rng.integers(0, 4, size=700).tolist()
+    w = synth.scaled(synth.CONFIGS[1], B=len(lens), V_ctc=33, dtype="bf16", seed=9, tau_ctc=1.5)
+    cb = synth.make_ctc_batch(w, "cpu", lens)
+    x = cb.logits.to(cuda_device)
+    out, gate = run_stage1(x, cb.frame_off, 33, 0, 2, 1.5, 2)
+    orc = H.oracle_stage1(H.storage_numpy(cb.logits), 33, cb.frame_off.numpy(), 0, 2, 1.5)
+    H.compare_stage1(out, gate, orc, cb.frame_off.numpy(), 1.5, require_all_margins=False)
+
+
+def test_thousands_of_utterances(cuda_device):
+    """A batch of 2,300 utterances of 0 to 8 frames."""
+    rng = np.random.default_rng(78)
+    lens = rng.integers(0, 9, size=2300).tolist()
+    w = synth.scaled(synth.CONFIGS[1], B=len(lens), V_ctc=129, dtype="f32", seed=10, tau_ctc=1.5)
+    cb = synth.make_ctc_batch(w, "cpu", lens)
+    x = cb.logits.to(cuda_device)
+    out, gate = run_stage1(x, cb.frame_off, 129, 0, 5, 1.5, 2)
+    orc = H.oracle_stage1(H.storage_numpy(cb.logits), 129, cb.frame_off.numpy(), 0, 5, 1.5)
+    H.compare_stage1(out, gate, orc, cb.frame_off.numpy(), 1.5, require_all_margins=False)
+
+
+def test_workspace_left_dirty_by_anything(cuda_device):
+    """The tile counter carries a per-call tag: whatever the workspace held before -- zeros, all
+    ones, the word of an earlier call -- and with no workspace at all (tiles dealt out in a
+    fixed order), the call gives the same outputs.  Few warps, so that most tiles are claimed
+    from the counter."""
+    dev = cuda_device
+    w = synth.scaled(synth.CONFIGS[1], B=6, seed=31)
+    cb = synth.make_ctc_batch(w, "cpu")
+    x, off = cb.logits.to(dev), cb.frame_off.to(dev)
+    ref_out = ssd.ssd_ctc_draft(x, off, 0, 200)
+    torch.cuda.synchronize()
+    few = H.opts(ctas=3, warps=2)
+    for fill in (0x00, 0xff, 0x5a, None):
+        out = ssd.alloc_ctc_outputs(x.shape[0], w.B, dev)
+        if fill is None:
+            del out["workspace"]
+        else:
+            out["workspace"].fill_(fill)
+        for _ in range(2):               # the second call finds the first call's word
+            ssd.ssd_ctc_draft(x, off, 0, 200, out=out, opts=few)
+            torch.cuda.synchronize()
+            for k in ("frame_entropy", "frame_argmax", "draft_len", "draft_full_len",
+                      "utt_max_entropy", "utt_status"):
+                assert torch.equal(out[k], ref_out[k]), (fill, k)
+            n = int(out["draft_len"].sum())
+            assert n > 0
+
+
+def test_internal_error_marks_never_pass_the_gate(cuda_device):
+    """The value a kernel leaves in a frame's entropy when one of its bounded waits ran out
+    (a NaN with a fixed payload) makes the gate refuse the utterance and report
+    SSD_UTT_INTERNAL; so does that status bit in the form that reads utterance maxima."""
+    dev = cuda_device
+    h = torch.full((10,), 0.01, dtype=torch.float32)
+    h[7] = torch.tensor([0x7fc0dead], dtype=torch.int32).view(torch.float32)[0]
+    off = torch.tensor([0, 5, 10], dtype=torch.int64)
+    gate = ssd.ssd_entropy_gate(h.to(dev), off.to(dev), 5.0)
+    assert gate["gate_accept"].cpu().tolist() == [1, 0]
+    mx = torch.tensor([0.01, 0.01, 0.01], dtype=torch.float32, device=dev)
+    st = torch.tensor([0, ssd.UTT_INTERNAL - (1 << 32), ssd.UTT_BAD_OFFSETS], dtype=torch.int32, device=dev)
+    g2 = ssd.ssd_entropy_gate_from_maxima(mx, st, 5.0)
+    assert g2["gate_accept"].cpu().tolist() == [1, 0, 0]
