@@ -6,9 +6,10 @@ ssd_verify) on synthetic logits shaped like the paper's workloads.
 
 A step is one pass of the whole path over one ragged batch.  One JSON line is printed by rank 0:
 utterances/s with the inputs resident in HBM, the same metric end to end from pinned host
-buffers, the HBM roofline fraction of the dominant kernel (timed with CUDA events recorded by
-the library around that kernel), the clocks seen under load, and the CPU oracle timed on the
-host cores as a reported baseline.  `--impl reference` times that oracle alone.
+buffers, the HBM roofline fraction of the streaming kernels (timed with CUDA events that the
+library records around them, on at least 24 launches whatever K is), the clocks seen under load,
+the CPU oracle timed on the host cores as a reported baseline, and the same figures for the
+other benchmark configurations in `per_config`.  `--impl reference` times that oracle alone.
 """
 import argparse
 import datetime
@@ -29,10 +30,11 @@ if ROOT not in sys.path:
 METRIC = "utterances/s for CTC draft+gate+verify"
 UNIT = "utterances/s"
 FALLBACK_HBM_GBS = 6650.0
-KERNEL_EVENT_EVERY = 5          # N_SETS and this are coprime: every input set gets timed
-N_SETS = 3                      # distinct input batches rotated through, so no step finds its
-                                # inputs in the 126 MB L2
-TRAFFIC_FILE = os.path.join(ROOT, "paper_2603_11243_b200", "ncu_traffic.json")
+NOMINAL_HBM_GBS = 8000.0        # the "~8 TB/s" the metric is stated against
+KERNEL_LAUNCHES = 24            # event-carrying launches per streaming kernel, after the timed region
+SMALL_SET_BYTES = 2e9           # below this, three input sets are rotated so that no step finds its
+                                # inputs in the 126 MB L2; above it one set is many times the L2
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "ncu_traffic.json")
 KERNEL_SOURCES = ["ssd_common.cuh", "ssd_stream.cuh", "ssd_ranges.cuh", "ssd_ctc.cu", "ssd_verify.cu",
                   "ssd_api.cu"]
 
@@ -40,14 +42,17 @@ KERNEL_SOURCES = ["ssd_common.cuh", "ssd_stream.cuh", "ssd_ranges.cuh", "ssd_ctc
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=3000)
-    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=1,
-                    help="workload index: 1..3 benchmark configurations; 5, 6 the paper's own "
-                         "shape at its high-accuracy / high-RTFx operating point")
-    ap.add_argument("--e2e-steps", type=int, default=30)
+    ap.add_argument("--config", type=int, default=3,
+                    help="workload index: 1..3 benchmark configurations (3, the largest that fits "
+                         "one GPU, is the headline); 5, 6 the paper's own shape at its "
+                         "high-accuracy / high-RTFx operating point")
+    ap.add_argument("--e2e-steps", type=int, default=0, help="0: 3 for workloads of more than 2 GB per step, else 30")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true",
+                    help="leave out the per_config records (the other benchmark configurations)")
     ap.add_argument("--verify-mode", default="full", choices=["full", "early_exit"],
                     help="full: ssd_verify reads every row of every verified utterance (the "
                          "benchmark metric); early_exit: ssd_verify_early_exit in its place, a "
@@ -57,13 +62,13 @@ def parse_args():
                          "JSON line per point to FILE instead of the benchmark line")
     ap.add_argument("--sweep-filter", default="", help="only points whose name contains this")
     ap.add_argument("--ncu-small", action="store_true",
-                    help="profiling aid: one input set, no end-to-end leg, no CPU baseline")
-    ap.add_argument("--ring-sweep", action="store_true",
-                    help="time ssd_verify's streaming kernel on --config for several stage sizes "
-                         "of its shared-memory ring (one JSON line each) instead of the benchmark")
+                    help="profiling aid: one input set, no end-to-end leg, no CPU baseline, no per_config")
     ap.add_argument("--ncu-stage1", action="store_true",
                     help="profiling aid: only the CTC batch of --config (a fraction of a GB even "
                          "where the whole step holds tens), ssd_ctc_draft three times, no timing")
+    ap.add_argument("--ncu-rows", type=int, default=0,
+                    help="profiling aid: ssd_verify alone on this many rows of --config's LLM "
+                         "vocabulary, three times, no timing")
     return ap.parse_args()
 
 
@@ -156,6 +161,10 @@ def summarise_clocks(rows, windows, note):
 
 
 # ---- our arm ---------------------------------------------------------------------------------
+def elem_size(w):
+    return 2 if w.dtype == "bf16" else 4
+
+
 def build_sets(w, device, n_sets, batch_lengths=None, verify_mode="full"):
     """Input sets and pre-marshalled calls.  The verify logits of a set have one row per draft
     token of the set's own CTC drafts (found by running stage 1 once, untimed).  With
@@ -176,8 +185,11 @@ def build_sets(w, device, n_sets, batch_lengths=None, verify_mode="full"):
         s1 = ssd.alloc_ctc_outputs(N, B, device)
         ssd.ssd_ctc_draft(cb.logits, off, wi.blank_id, wi.max_draft_len, out=s1)
         gate = ssd.alloc_gate_outputs(B, device)
+        # the gate's first form once, as a check of the form the timed steps use
         ssd.ssd_entropy_gate(s1["frame_entropy"], off, wi.tau_ctc, out=gate)
+        g2 = ssd.ssd_entropy_gate_from_maxima(s1["utt_max_entropy"], s1["utt_status"], wi.tau_ctc)
         torch.cuda.synchronize()
+        assert torch.equal(g2["gate_accept"], gate["gate_accept"]), "the two forms of the gate disagree"
         K = s1["draft_len"].cpu().tolist()
         vb = synth.make_verify_batch(wi, K, device)
         M = vb.logits.shape[0]
@@ -186,7 +198,7 @@ def build_sets(w, device, n_sets, batch_lengths=None, verify_mode="full"):
         s2 = ssd.alloc_verify_outputs(M, B, device, ssd.ssd_verify_workspace_bytes(B, M, wi.V_llm, code))
         skipped = gate["gate_accept"].cpu().numpy().astype(bool)
         m_active = int(sum(k for k, s in zip(K, skipped) if not s))
-        es = 2 if wi.dtype == "bf16" else 4
+        es = elem_size(wi)
         if verify_mode == "early_exit":
             # the full call first (its decisions are the check), then the early-exit one, whose
             # rows_read give the bytes this mode really reads
@@ -209,9 +221,19 @@ def build_sets(w, device, n_sets, batch_lengths=None, verify_mode="full"):
             B=B, N=N, M=M, K=K, m_active=m_active,
             ctc_bytes=N * wi.V_ctc * es, verify_bytes=m_active * wi.V_llm * es,
             call_ctc=ssd.bind_ctc_draft(cb.logits, off, wi.blank_id, wi.max_draft_len, s1),
-            call_gate=ssd.bind_entropy_gate(s1["frame_entropy"], off, wi.tau_ctc, gate),
+            call_gate=ssd.bind_entropy_gate_from_maxima(s1["utt_max_entropy"], s1["utt_status"],
+                                                        wi.tau_ctc, gate),
             call_verify=call_verify))
     return sets
+
+
+def step(s, o_ctc=None, o_ver=None):
+    """One pass of the path over one batch: frame statistics and collapse (Eq. 2, Section 2.1),
+    the entropy gate (Eq. 3; from the utterance maxima the first call left), verification of
+    the utterances the gate did not accept (Eq. 5, Section 2.3)."""
+    s["call_ctc"](o_ctc)
+    s["call_gate"]()
+    s["call_verify"](o_ver)
 
 
 def make_events(n):
@@ -222,6 +244,158 @@ def make_events(n):
         e.record()
     torch.cuda.synchronize()
     return evs
+
+
+def time_kernels(sets, launches=KERNEL_LAUNCHES):
+    """Durations (ms) of the two streaming kernels over `launches` further steps, each step
+    carrying the events the library records just around those kernels.  (An event between two
+    kernels keeps the second from being scheduled early, so the steps of the timed region carry
+    none.)"""
+    import torch
+    from paper_2603_11243_b200 import binding as ssd
+    n_sets = len(sets)
+    ev = make_events(4 * launches)
+    for j in range(launches):
+        a, b = ssd.LaunchOpts(), ssd.LaunchOpts()
+        a.ev_begin, a.ev_end = ev[4 * j].cuda_event, ev[4 * j + 1].cuda_event
+        b.ev_begin, b.ev_end = ev[4 * j + 2].cuda_event, ev[4 * j + 3].cuda_event
+        step(sets[j % n_sets], a, b)
+    torch.cuda.synchronize()
+    t_ctc = [ev[4 * j].elapsed_time(ev[4 * j + 1]) for j in range(launches)]
+    t_ver = [ev[4 * j + 2].elapsed_time(ev[4 * j + 3]) for j in range(launches)]
+    ctc_bytes = statistics.mean(sets[j % n_sets]["ctc_bytes"] for j in range(launches))
+    ver_bytes = statistics.mean(sets[j % n_sets]["verify_bytes"] for j in range(launches))
+    return t_ctc, t_ver, ctc_bytes, ver_bytes
+
+
+def roof(kernel, nbytes, times_ms, peak, peak_kind):
+    """Roofline record of one streaming kernel: algorithmic bytes per launch over the mean
+    launch duration (median and best beside it), against the measured copy bandwidth and against
+    the nominal 8 TB/s."""
+    times = [t for t in times_ms if t > 0]
+    if not times or nbytes <= 0:
+        return {"kernel": kernel, "bound": "hbm", "achieved": 0.0, "peak": peak, "unit": "GB/s",
+                "frac": 0.0, "peak_kind": "of " + peak_kind, "traffic": None,
+                "algorithmic_bytes_per_launch": int(nbytes), "launches_timed": len(times),
+                "note": "nothing to read in this configuration"}
+    avg, med, best = statistics.mean(times), statistics.median(times), min(times)
+    gbs = lambda ms: nbytes / (ms * 1e-3) / 1e9
+    return {"kernel": kernel, "bound": "hbm", "achieved": round(gbs(avg), 1), "peak": peak,
+            "unit": "GB/s", "frac": round(gbs(avg) / peak, 4), "peak_kind": "of " + peak_kind,
+            "frac_median": round(gbs(med) / peak, 4), "frac_best": round(gbs(best) / peak, 4),
+            "frac_of_nominal": round(gbs(avg) / NOMINAL_HBM_GBS, 4), "nominal_peak": NOMINAL_HBM_GBS,
+            "traffic": recorded_traffic(kernel, nbytes),
+            "algorithmic_bytes_per_launch": int(nbytes), "launches_timed": len(times),
+            "avg_launch_us": round(avg * 1e3, 2), "median_launch_us": round(med * 1e3, 2),
+            "min_launch_us": round(best * 1e3, 2)}
+
+
+def timed_steps(sets, K, W, barrier=None):
+    """W warm-up steps, then K steps between two events with a synchronize on both sides.
+    Returns (ms for the K steps, wall-clock window, kernels launched in the window)."""
+    import torch
+    from paper_2603_11243_b200 import binding as ssd
+    n_sets = len(sets)
+    for i in range(W):
+        step(sets[i % n_sets])
+    torch.cuda.synchronize()
+    ev = make_events(2)
+    if barrier:
+        barrier()
+    torch.cuda.synchronize()
+    wall0 = time.time()
+    l0 = int(ssd.lib().ssd_launch_count())
+    ev[0].record()
+    for i in range(K):
+        step(sets[i % n_sets])
+    ev[1].record()
+    torch.cuda.synchronize()
+    wall1 = time.time()
+    launches = int(ssd.lib().ssd_launch_count()) - l0
+    if barrier:
+        barrier()
+    return ev[0].elapsed_time(ev[1]), (wall0, wall1), launches
+
+
+def sets_for(w, device, verify_mode="full", one_set=False):
+    from paper_2603_11243_b200 import synth
+    batch_lengths = None
+    est = w.B * (0.5 * (w.t_lo + w.t_hi) * w.V_ctc + min(w.max_draft_len, 0.2 * (w.t_lo + w.t_hi)) * w.V_llm) * elem_size(w)
+    n_sets = 1 if (one_set or est > SMALL_SET_BYTES) else 3
+    if w.name.startswith("paper_"):
+        # the paper's batching: a pool of utterances, length-sorted, <= 50,000 frames per batch
+        batch_lengths = synth.length_sorted_batches(synth.draw_lengths(w))
+        n_sets = 1 if one_set else len(batch_lengths)
+    return build_sets(w, device, n_sets, batch_lengths, verify_mode), batch_lengths
+
+
+def l2_note(sets):
+    s0 = sets[0]
+    per_set = s0["ctc_bytes"] + s0["M"] * s0["w"].V_llm * elem_size(s0["w"])
+    if len(sets) > 1:
+        return ("inputs larger than L2: %d distinct input batches of %.2f GB rotated" %
+                (len(sets), per_set / 1e9))
+    return "inputs larger than L2: one input batch of %.2f GB, %d times the 126 MB L2" % (
+        per_set / 1e9, int(per_set / 126e6))
+
+
+def workload_string(idx, base, w, batch_lengths):
+    return ("configs[%s] %s: B=%s utterances per GPU, T~%s[%d,%d], V_ctc=%d, V_llm=%d, "
+            "draft_len<=%d, %s logits (fp32 accumulation)" %
+            (idx, base.name,
+             w.B if batch_lengths is None else
+             "%d in %d length-sorted batches of <=50,000 frames; a step is one batch;"
+             % (w.B, len(batch_lengths)),
+             w.t_dist, w.t_lo, w.t_hi, w.V_ctc, w.V_llm, w.max_draft_len, w.dtype))
+
+
+PER_CONFIG = [("configs[1]", 1, None), ("configs[2]", 2, None),
+              ("configs[4] B=64 V_llm=49152 bf16", 4, (64, 49152, "bf16")),
+              ("configs[4] B=64 V_llm=152064 bf16", 4, (64, 152064, "bf16")),
+              ("configs[4] B=64 V_llm=49152 f32", 4, (64, 49152, "f32")),
+              ("configs[4] B=64 V_llm=152064 f32", 4, (64, 152064, "f32")),
+              ("configs[4] B=1024 V_llm=49152 bf16", 4, (1024, 49152, "bf16")),
+              ("configs[4] B=1024 V_llm=49152 f32", 4, (1024, 49152, "f32")),
+              ("configs[4] B=1 V_llm=32000 bf16", 4, (1, 32000, "bf16")),
+              ("configs[4] B=1 V_llm=152064 f32", 4, (1, 152064, "f32"))]
+
+
+def run_per_config(device, peak, peak_kind, skip_idx, cpu=True):
+    """The other benchmark configurations, each timed like the headline (fewer steps): whole-step
+    throughput, both streaming kernels on KERNEL_LAUNCHES event-carrying launches, the oracle on
+    a bounded sample."""
+    import torch
+    from paper_2603_11243_b200 import synth
+    out = {}
+    for name, idx, point in PER_CONFIG:
+        if idx == skip_idx and point is None:
+            continue
+        w = synth.CONFIGS[idx] if point is None else synth.sweep_point(*point)
+        t0 = time.time()
+        sets, _ = sets_for(w, device)
+        est_ms = max(0.02, sum(s["ctc_bytes"] + s["verify_bytes"] for s in sets) / len(sets) / 5e9)
+        K = int(max(20, min(400, 60.0 / est_ms)))
+        ms, _, launches = timed_steps(sets, K, 5)
+        t_ctc, t_ver, ctc_b, ver_b = time_kernels(sets)
+        units = sum(sets[i % len(sets)]["B"] for i in range(K))
+        step_bytes = statistics.mean(s["ctc_bytes"] + s["verify_bytes"] for s in sets)
+        rec = {"workload": workload_string(idx, w, w, None), "steps": K,
+               "value": round(units / (ms * 1e-3), 1), "unit": UNIT,
+               "ms_per_step": round(ms / K, 5), "gpu_launches_per_step": launches / K,
+               "logits_bytes_per_step": int(step_bytes),
+               "step_hbm_gbs": round(step_bytes / (ms / K * 1e-3) / 1e9, 1),
+               "step_frac_of_peak": round(step_bytes / (ms / K * 1e-3) / 1e9 / peak, 4),
+               "step_frac_of_nominal": round(step_bytes / (ms / K * 1e-3) / 1e9 / NOMINAL_HBM_GBS, 4),
+               "l2": l2_note(sets),
+               "roofline_ctc": roof("ctc_rows_tma", ctc_b, t_ctc, peak, peak_kind),
+               "roofline_verify": roof("verify_rows_tma", ver_b, t_ver, peak, peak_kind)}
+        if cpu:
+            rec["cpu_baseline"] = cpu_baseline(sets[0], budget_s=2.5)
+        rec["seconds_spent"] = round(time.time() - t0, 1)
+        out[name] = rec
+        del sets
+        torch.cuda.empty_cache()
+    return out
 
 
 def run_ours(args):
@@ -243,51 +417,15 @@ def run_ours(args):
 
     base = synth.CONFIGS[args.config]
     w = synth.scaled(base, seed=D.rank_seed(base.seed, rank))
-    n_sets = 1 if args.ncu_small else N_SETS
-    batch_lengths = None
-    if args.config >= 5:
-        # the paper's batching: a pool of utterances, length-sorted, <= 50,000 frames per batch
-        batch_lengths = synth.length_sorted_batches(synth.draw_lengths(w))
-        n_sets = 1 if args.ncu_small else len(batch_lengths)
-    sets = build_sets(w, device, n_sets, batch_lengths, args.verify_mode)
+    sets, batch_lengths = sets_for(w, device, args.verify_mode, one_set=args.ncu_small)
+    n_sets = len(sets)
     K, W = args.steps, args.warmup
 
-    def step(s, o_ctc=None, o_ver=None):
-        s["call_ctc"](o_ctc)
-        s["call_gate"]()
-        s["call_verify"](o_ver)
-
-    for i in range(W):
-        step(sets[i % n_sets])
-    torch.cuda.synchronize()
-
-    # ---- timed region: K steps, inputs resident in HBM -------------------------------------
-    # Per-kernel durations come from events the library records around its streaming kernel.
-    # An event between two kernels keeps the second from being scheduled early, so only every
-    # KERNEL_EVENT_EVERY-th step of the timed region carries them.
-    timed_steps = list(range(0, K, KERNEL_EVENT_EVERY))
-    ev = make_events(4 * len(timed_steps) + 2)
-    opts_ctc, opts_ver = [None] * K, [None] * K
-    for j, i in enumerate(timed_steps):
-        a, b = ssd.LaunchOpts(), ssd.LaunchOpts()
-        a.ev_begin, a.ev_end = ev[4 * j].cuda_event, ev[4 * j + 1].cuda_event
-        b.ev_begin, b.ev_end = ev[4 * j + 2].cuda_event, ev[4 * j + 3].cuda_event
-        opts_ctc[i], opts_ver[i] = a, b
-    t_begin, t_end = ev[-2], ev[-1]
+    # ---- timed region: W warm-up steps, then K steps with the inputs resident in HBM ---------
     sampler = ClockSampler(local_rank) if rank == 0 else None
-    D.barrier()
-    torch.cuda.synchronize()
-    wall0 = time.time()
-    t_begin.record()
-    for i in range(K):
-        step(sets[i % n_sets], opts_ctc[i], opts_ver[i])
-    t_end.record()
-    torch.cuda.synchronize()
-    wall1 = time.time()
-    D.barrier()
-    ms_total = t_begin.elapsed_time(t_end)
-    windows, clock_note = [(wall0, wall1)], "timed region"
-    if rank == 0 and wall1 - wall0 < 0.6 and not args.ncu_small:
+    ms_total, window, launches = timed_steps(sets, K, W, barrier=D.barrier)
+    windows, clock_note = [window], "timed region"
+    if rank == 0 and window[1] - window[0] < 0.6 and not args.ncu_small:
         # the region is too short for a 50 ms sampler: keep the same load up a little longer
         wall2 = time.time()
         i = 0
@@ -304,30 +442,19 @@ def run_ours(args):
     ms_max, units = D.reduce_max_sum(ms_total, float(sum(sets[i % n_sets]["B"] for i in range(K))),
                                      device)
     value = units / (ms_max * 1e-3)
-
-    t_ctc = [ev[4 * j].elapsed_time(ev[4 * j + 1]) for j in range(len(timed_steps))]
-    t_ver = [ev[4 * j + 2].elapsed_time(ev[4 * j + 3]) for j in range(len(timed_steps))]
-    ctc_bytes = statistics.mean(sets[i % n_sets]["ctc_bytes"] for i in timed_steps)
-    ver_bytes = statistics.mean(sets[i % n_sets]["verify_bytes"] for i in timed_steps)
     step_bytes = statistics.mean(sets[i % n_sets]["ctc_bytes"] + sets[i % n_sets]["verify_bytes"]
                                  for i in range(K))
     peak, peak_kind = peaks()
 
+    # ---- the streaming kernels alone, on KERNEL_LAUNCHES further steps that carry events ------
+    t_ctc, t_ver, ctc_bytes, ver_bytes = time_kernels(sets, 3 if args.ncu_small else KERNEL_LAUNCHES)
     vkern = "verify_rows_tma" if args.verify_mode == "full" else "verify_rows_ee"
-
-    def roof(kernel, nbytes, times_ms):
-        avg = statistics.mean(times_ms)
-        ach = nbytes / (avg * 1e-3) / 1e9 if avg > 0 else 0.0
-        return {"kernel": kernel, "bound": "hbm", "achieved": round(ach, 1), "peak": peak,
-                "unit": "GB/s", "frac": round(ach / peak, 4), "peak_kind": "of " + peak_kind,
-                "traffic": recorded_traffic(kernel, nbytes),
-                "algorithmic_bytes_per_launch": int(nbytes), "launches_timed": len(times_ms),
-                "avg_launch_us": round(avg * 1e3, 2), "min_launch_us": round(min(times_ms) * 1e3, 2)}
 
     # ---- end to end: pinned host buffers in, decisions out, every step ---------------------
     e2e = None
     if not args.ncu_small:
-        e2e = run_e2e(sets[0], device, args.e2e_steps, D, world)
+        e2e_steps = args.e2e_steps or (3 if step_bytes > 2e9 else 30)
+        e2e = run_e2e(sets[0], device, e2e_steps, D, world)
 
     if rank != 0:
         D.finalize()
@@ -338,35 +465,31 @@ def run_ours(args):
     gate_acc = float(s0["gate"]["gate_accept"].float().mean().item())
     all_acc = s0["s2"]["all_accepted"].cpu().numpy().astype(bool)
     skipped = s0["gate"]["gate_accept"].cpu().numpy().astype(bool)
+    r_ctc = roof("ctc_rows_tma", ctc_bytes, t_ctc, peak, peak_kind)
+    r_ver = roof(vkern, ver_bytes, t_ver, peak, peak_kind)
     line = {
         "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": K,
         "warmup": W, "ms_per_step": round(ms_max / K, 5), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {
-            "workload": "configs[%d] %s: B=%s utterances per GPU, T~%s[%d,%d], V_ctc=%d, "
-                        "V_llm=%d, draft_len<=%d, %s logits (fp32 accumulation)" %
-                        (args.config, base.name,
-                         w.B if batch_lengths is None else
-                         "%d in %d length-sorted batches of <=50,000 frames; a step is one batch;"
-                         % (w.B, len(batch_lengths)),
-                         w.t_dist, w.t_lo, w.t_hi, w.V_ctc, w.V_llm, w.max_draft_len, w.dtype),
+            "workload": workload_string(args.config, base, w, batch_lengths),
+            "logits_dtype": w.dtype, "accumulation_dtype": "f32",
             "generator": w.variant, "tau_ctc": w.tau_ctc, "tau_slm": w.tau_slm,
             "verify_mode": args.verify_mode,
+            "calls_per_step": "ssd_ctc_draft, ssd_entropy_gate (from the utterance maxima), ssd_verify",
             "frames_per_step": s0["N"], "verify_rows_per_step": s0["M"],
             "verify_rows_read_per_step": s0["m_active"],
             "logits_bytes_per_step": int(step_bytes),
-            "l2": "inputs larger than L2: %d distinct input batches of %.2f GB rotated, each "
-                  "step reads %.2f GB once" % (n_sets, (s0["ctc_bytes"] + s0["M"] * w.V_llm * 2) / 1e9,
-                                              step_bytes / 1e9),
+            "l2": l2_note(sets) + "; each step reads %.2f GB once" % (step_bytes / 1e9),
             "parallelism": "utterances sharded over %d rank(s), no data-path collective" % world},
-        "gpu_launches": (5 if args.verify_mode == "full" else 6) * K,
+        "gpu_launches": launches,
         # `roofline` is the kernel that holds most of the step's device time
-        "roofline": roof(vkern, ver_bytes, t_ver) if sum(t_ver) >= sum(t_ctc)
-                    else roof("ctc_rows_tma", ctc_bytes, t_ctc),
-        "roofline_ctc": roof("ctc_rows_tma", ctc_bytes, t_ctc),
-        "roofline_verify": roof(vkern, ver_bytes, t_ver),
+        "roofline": r_ver if sum(t_ver) >= sum(t_ctc) else r_ctc,
+        "roofline_ctc": r_ctc,
+        "roofline_verify": r_ver,
         "step_hbm_gbs": round(step_bytes / (ms_max / K * 1e-3) / 1e9, 1),
         "step_frac_of_peak": round(step_bytes / (ms_max / K * 1e-3) / 1e9 / peak, 4),
+        "step_frac_of_nominal": round(step_bytes / (ms_max / K * 1e-3) / 1e9 / NOMINAL_HBM_GBS, 4),
         "decisions": {"gate_accept_frac": round(gate_acc, 4),
                       "verify_all_accepted_frac_of_verified":
                           round(float(all_acc[~skipped].mean()) if (~skipped).any() else 0.0, 4)},
@@ -375,7 +498,12 @@ def run_ours(args):
         "next_rows": next_rows,
     }
     if world == 1 and not args.no_cpu_baseline and not args.ncu_small:
-        line["cpu_baseline"] = cpu_baseline(s0, budget_s=20.0)
+        line["cpu_baseline"] = cpu_baseline(s0, budget_s=16.0, single_thread_too=True)
+    del sets
+    torch.cuda.empty_cache()
+    if world == 1 and not args.ncu_small and not args.no_per_config:
+        line["per_config"] = run_per_config(device, peak, peak_kind, args.config,
+                                            cpu=not args.no_cpu_baseline)
     print(json.dumps(line), flush=True)
     D.finalize()
 
@@ -423,15 +551,15 @@ def time_next_rows(sets, device, peak):
         sets[i]["s2"]["accepted_len"], sets[i]["s2"]["all_accepted"], out=prep[i][1]))
     t_gr = timed(lambda i: ssd.ssd_greedy_step(sets[i]["vb"].logits[:R], out=prep[i][2]))
     # the streaming kernel alone, from events the library records around it
-    kev = make_events(2 * 12)
-    for j in range(12):
+    kev = make_events(2 * KERNEL_LAUNCHES)
+    for j in range(KERNEL_LAUNCHES):
         o = ssd.LaunchOpts()
         o.ev_begin, o.ev_end = kev[2 * j].cuda_event, kev[2 * j + 1].cuda_event
         ssd.ssd_greedy_step(sets[j % n_sets]["vb"].logits[:R], out=prep[j % n_sets][2], opts=o)
     torch.cuda.synchronize()
-    t_gk = statistics.mean(kev[2 * j].elapsed_time(kev[2 * j + 1]) for j in range(2, 12)) * 1e3
+    t_gk = statistics.mean(kev[2 * j].elapsed_time(kev[2 * j + 1]) for j in range(2, KERNEL_LAUNCHES)) * 1e3
     w = sets[0]["w"]
-    gbytes = R * w.V_llm * (2 if w.dtype == "bf16" else 4)
+    gbytes = R * w.V_llm * elem_size(w)
     # the whole step with ssd_verify_early_exit in place of ssd_verify (same decisions; the
     # per-token log-likelihoods only up to a little past each first reject)
     code = ssd.BF16 if w.dtype == "bf16" else ssd.F32
@@ -460,6 +588,7 @@ def time_next_rows(sets, device, peak):
              "same_decisions_as_full": bool(same),
              "note": "separate mode, not part of `value`: rows after an utterance's first reject "
                      "are not read (Section 2.3 needs only the first reject)"}
+    del ee
     # one rank's share of a vocabulary-parallel head: a quarter of the columns, then the
     # combination of four ranks' statistics (this GPU's own four slices stand in for them; the
     # all-gather between ranks, 12 bytes per row, needs more than one GPU and is not timed)
@@ -488,13 +617,14 @@ def time_next_rows(sets, device, peak):
         t_cb = timed(lambda i: ssd.ssd_verify_combine(
             vsh[i][1], w.V_llm, sets[i]["tok_off"], sets[i]["ids"], w.tau_slm,
             skip=sets[i]["gate"]["gate_accept"], out=vsh[i][2]))
-        sh_bytes = rows_full / n_sets * vq * (2 if w.dtype == "bf16" else 4)
+        sh_bytes = rows_full / n_sets * vq * elem_size(w)
         vp = {"ranks": 4, "shard_us": round(t_sh, 2), "combine_us": round(t_cb, 2),
               "shard_gbs": round(sh_bytes / (t_sh * 1e-6) / 1e9, 1),
               "same_decisions_as_full": bool(same_vp),
               "note": "ssd_verify_shard on columns [V/4, V/2) (host-paced call: streaming kernel "
                       "plus its closing kernel) and ssd_verify_combine over four slices' "
                       "statistics; the all-gather between ranks is not part of it"}
+        del vsh
     return {"early_exit_step": early, "vocab_parallel_verify": vp,
             "threshold_sweep": {"pairs": len(pairs), "us_per_call": round(t_sw, 2)},
             "assemble": {"us_per_call": round(t_asm, 2),
@@ -514,7 +644,11 @@ def run_e2e(s, device, steps, D, world):
     calls and reads the per-utterance decisions and the draft back to the host."""
     import torch
     w = s["w"]
-    pin = lambda t: t.detach().cpu().contiguous().pin_memory()
+
+    def pin(t):
+        h = torch.empty(t.shape, dtype=t.dtype, pin_memory=True)
+        h.copy_(t)
+        return h
     h_in = dict(ctc=pin(s["cb"].logits), llm=pin(s["vb"].logits), off=pin(s["off"]),
                 tok_off=pin(s["tok_off"]), ids=pin(s["ids"]))
     d_in = dict(ctc=s["cb"].logits, llm=s["vb"].logits, off=s["off"], tok_off=s["tok_off"],
@@ -529,14 +663,12 @@ def run_e2e(s, device, steps, D, world):
     def one():
         for k in h_in:
             d_in[k].copy_(h_in[k], non_blocking=True)
-        s["call_ctc"]()
-        s["call_gate"]()
-        s["call_verify"]()
+        step(s)
         for d, h in zip(outs, h_out):
             h.copy_(d, non_blocking=True)
         torch.cuda.current_stream().synchronize()      # the caller reads the decisions now
 
-    for _ in range(3):
+    for _ in range(1 if h2d > 2e9 else 3):
         one()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     D.barrier()
@@ -552,15 +684,18 @@ def run_e2e(s, device, steps, D, world):
     # host waits are part of this number: take the larger of device and wall time
     sec = max(e0.elapsed_time(e1) * 1e-3, wall)
     sec_max, units = D.reduce_max_sum(sec, float(steps * s["B"]), device)
+    del h_in
     return {"value": round(units / sec_max, 1), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
             "d2h_bytes_per_step": int(d2h), "steps": steps,
             "ms_per_step": round(sec_max / steps * 1e3, 4),
+            "h2d_gbs": round(h2d * steps / sec_max / 1e9, 1),
             "note": "pinned host -> device copies of all logits, three C-ABI calls, decisions "
                     "and draft copied back, stream synchronised every step"}
 
 
 # ---- the oracle as a CPU baseline ------------------------------------------------------------
-def host_inputs(s):
+def host_inputs(s, n_utt):
+    """Host copies (in the form the oracle takes) of the first n_utt utterances of a batch."""
     import numpy as np
     import torch
 
@@ -569,9 +704,10 @@ def host_inputs(s):
         if t.dtype == torch.bfloat16:
             return t.view(torch.int16).numpy().view(np.uint16)
         return t.numpy()
-    return dict(ctc=to_np(s["cb"].logits), llm=to_np(s["vb"].logits),
-                off=s["cb"].frame_off.numpy(), tok_off=s["vb"].tok_off.numpy(),
-                ids=s["vb"].draft_ids.numpy())
+    off, tok = s["cb"].frame_off.numpy(), s["vb"].tok_off.numpy()
+    f1, k1 = int(off[n_utt]), int(tok[n_utt])
+    return dict(ctc=to_np(s["cb"].logits[:f1]), llm=to_np(s["vb"].logits[:k1]),
+                off=off[:n_utt + 1], tok_off=tok[:n_utt + 1], ids=s["vb"].draft_ids.numpy()[:k1])
 
 
 def oracle_pass(h, w, lo, hi):
@@ -588,23 +724,35 @@ def oracle_pass(h, w, lo, hi):
     return time.perf_counter() - t0
 
 
-def cpu_baseline(s, budget_s):
+def cpu_baseline(s, budget_s, single_thread_too=False):
     """The oracle as it stands on the host cores, one utterance per thread, on a bounded sample:
-    the batch (or its first utterances) repeated until about `budget_s` core-seconds are spent."""
+    the first utterances of the batch, as many as about `budget_s` seconds of wall time allow
+    (at least one per thread).  With single_thread_too, one thread on a few utterances as well."""
     from oracle import ref
     w = s["w"]
     cores = len(os.sched_getaffinity(0))
     threads = ref.set_threads(max(1, min(cores, w.B)))
-    h = host_inputs(s)
-    t1 = oracle_pass(h, w, 0, min(w.B, threads))            # one utterance per thread
-    core_s_per_utt = t1                      # each thread worked t1 seconds on one utterance
-    n = int(min(w.B, max(threads, budget_s / max(core_s_per_utt, 1e-9))))
-    reps = int(max(1, min(50, round(budget_s / max(core_s_per_utt * n, 1e-9)))))
+    first = min(w.B, threads)
+    h = host_inputs(s, first)
+    t1 = oracle_pass(h, w, 0, first)            # one utterance per thread
+    n = int(min(w.B, max(first, first * budget_s / max(t1, 1e-9))))
+    n -= n % threads if n > threads else 0
+    if n > first:
+        h = host_inputs(s, n)
+    reps = int(max(1, min(50, round(budget_s / max(t1 * n / first, 1e-9)))))
     sec = sum(oracle_pass(h, w, 0, n) for _ in range(reps))
-    return {"value": round(n * reps / sec, 2), "unit": UNIT, "cores": threads, "kind": "oracle",
-            "sample": "first %d of the %d utterances of one batch, whole path (fp64 two-pass C "
-                      "oracle, one utterance per thread), %d pass(es), %.1f s wall = %.0f "
-                      "core-seconds" % (n, w.B, reps, sec, sec * threads)}
+    rec = {"value": round(n * reps / sec, 2), "unit": UNIT, "cores": threads, "kind": "oracle",
+           "sample": "first %d of the %d utterances of one batch, whole path (fp64 two-pass C "
+                     "oracle, one utterance per thread), %d pass(es), %.1f s wall = %.0f "
+                     "core-seconds" % (n, w.B, reps, sec, sec * threads)}
+    if single_thread_too:
+        ref.set_threads(1)
+        m = max(1, min(n, int(round(0.25 * budget_s / max(t1, 1e-9)))))   # t1 ~ one utterance on one core
+        sec1 = oracle_pass(h, w, 0, m)
+        ref.set_threads(threads)
+        rec["single_thread"] = {"value": round(m / sec1, 2), "unit": UNIT, "cores": 1,
+                                "sample": "first %d utterance(s), %.1f s" % (m, sec1)}
+    return rec
 
 
 def run_reference(args):
@@ -612,29 +760,34 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
+    import numpy as np
     import torch
     from oracle import ref
     from paper_2603_11243_b200 import synth
-    w = synth.CONFIGS[args.config]
+    base = synth.CONFIGS[args.config]
     K, W = args.steps, args.warmup
-    dev = "cpu"
-    cb = synth.make_ctc_batch(w, dev)
-    # the oracle's own drafts size the verify batch, as the GPU arm's drafts size its batch
-    import numpy as np
+    cores = len(os.sched_getaffinity(0))
+    threads = ref.set_threads(max(1, min(cores, base.B)))
+    # The oracle sees a bounded sample of the workload: a smaller batch of the same configuration
+    # (same generators and value mix, fewer utterances), since it could not get through the full
+    # batch of the larger configurations in minutes.
+    pool = int(min(base.B, 2 * threads))
+    w = synth.scaled(base, B=pool)
+
     def to_np(t):
         t = t.contiguous()
         return t.view(torch.int16).numpy().view(np.uint16) if t.dtype == torch.bfloat16 else t.numpy()
+    cb = synth.make_ctc_batch(w, "cpu")
     ctc = to_np(cb.logits)
-    cores = len(os.sched_getaffinity(0))
-    threads = ref.set_threads(max(1, min(cores, w.B)))
+    # the oracle's own drafts size the verify batch, as the GPU arm's drafts size its batch
     o1 = ref.ctc_draft(ctc, w.V_ctc, cb.frame_off.numpy(), w.blank_id, w.max_draft_len)
-    vb = synth.make_verify_batch(w, o1["draft_len"].tolist(), dev)
+    vb = synth.make_verify_batch(w, o1["draft_len"].tolist(), "cpu")
     h = dict(ctc=ctc, llm=to_np(vb.logits), off=cb.frame_off.numpy(), tok_off=vb.tok_off.numpy(),
              ids=vb.draft_ids.numpy())
     # bounded sample per step: u utterances, sized so that K + W steps take about two minutes
-    probe = oracle_pass(h, w, 0, min(w.B, threads)) / min(w.B, threads)
-    u = int(max(1, min(w.B, 120.0 / max(K + W, 1) / max(probe, 1e-9))))
-    starts = [(i * u) % max(1, w.B - u + 1) for i in range(K + W)]
+    probe = oracle_pass(h, w, 0, min(pool, threads)) / min(pool, threads)
+    u = int(max(1, min(pool, 100.0 / max(K + W, 1) / max(probe, 1e-9))))
+    starts = [(i * u) % max(1, pool - u + 1) for i in range(K + W)]
     for i in range(W):
         oracle_pass(h, w, starts[i], starts[i] + u)
     t0 = time.perf_counter()
@@ -642,14 +795,15 @@ def run_reference(args):
         oracle_pass(h, w, starts[i], starts[i] + u)
     sec = time.perf_counter() - t0
     value = K * u / sec
-    sample = ("%d utterance(s) of the configs[%d] batch per step (window sliding over the batch), "
-              "whole path in the fp64 C oracle, %d thread(s)" % (u, args.config, threads))
+    sample = ("%d utterance(s) per step out of a %d-utterance batch of configs[%d] (window "
+              "sliding over them), whole path in the fp64 C oracle, %d thread(s)" %
+              (u, pool, args.config, threads))
     line = {"impl": "reference", "metric": METRIC, "value": round(value, 3), "unit": UNIT,
             "n_gpus": args.gpus, "steps": K, "warmup": W, "ms_per_step": round(sec / K * 1e3, 3),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
             "data": "synthetic",
             "config": {"workload": "configs[%d] %s (CPU oracle on a bounded sample per step)" %
-                                   (args.config, w.name), "sample": sample},
+                                   (args.config, base.name), "sample": sample},
             "cpu_baseline": {"value": round(value, 3), "unit": UNIT, "cores": threads,
                              "kind": "oracle", "sample": sample},
             "e2e": {"value": round(value, 3), "unit": UNIT, "h2d_bytes_per_step": 0,
@@ -664,39 +818,6 @@ SWEEP_V = (32000, 49152, 100352, 152064)
 SWEEP_DTYPES = ("f32", "bf16")
 SWEEP_MAX_RESIDENT = 48e9        # bytes of logits generated at a time; larger points run as
                                  # equal sub-batches, each timed on its own, times added
-
-
-def time_steps(sets, steps, warmup, every=3):
-    """Mean step time and mean streaming-kernel times (ms) over `steps` steps."""
-    import torch
-    from paper_2603_11243_b200 import binding as ssd
-    n_sets = len(sets)
-
-    def step(s, o_ctc=None, o_ver=None):
-        s["call_ctc"](o_ctc)
-        s["call_gate"]()
-        s["call_verify"](o_ver)
-
-    for i in range(warmup):
-        step(sets[i % n_sets])
-    timed = list(range(0, steps, every))
-    ev = make_events(4 * len(timed) + 2)
-    opts = {}
-    for j, i in enumerate(timed):
-        a, b = ssd.LaunchOpts(), ssd.LaunchOpts()
-        a.ev_begin, a.ev_end = ev[4 * j].cuda_event, ev[4 * j + 1].cuda_event
-        b.ev_begin, b.ev_end = ev[4 * j + 2].cuda_event, ev[4 * j + 3].cuda_event
-        opts[i] = (a, b)
-    torch.cuda.synchronize()
-    ev[-2].record()
-    for i in range(steps):
-        o = opts.get(i, (None, None))
-        step(sets[i % n_sets], o[0], o[1])
-    ev[-1].record()
-    torch.cuda.synchronize()
-    t_ctc = statistics.mean(ev[4 * j].elapsed_time(ev[4 * j + 1]) for j in range(len(timed)))
-    t_ver = statistics.mean(ev[4 * j + 2].elapsed_time(ev[4 * j + 3]) for j in range(len(timed)))
-    return ev[-2].elapsed_time(ev[-1]) / steps, t_ctc, t_ver
 
 
 def run_sweep(args):
@@ -714,7 +835,7 @@ def run_sweep(args):
                     w = synth.sweep_point(B, V, dtype)
                     if args.sweep_filter and args.sweep_filter not in w.name:
                         continue
-                    es = 2 if dtype == "bf16" else 4
+                    es = elem_size(w)
                     est = B * (1000 * w.V_ctc + 250 * V) * es
                     n_sub = max(1, math.ceil(est / SWEEP_MAX_RESIDENT))
                     while B % n_sub:
@@ -723,19 +844,23 @@ def run_sweep(args):
                     steps = int(max(10, min(300, 0.25 / (est / n_sub / 5e12))))
                     ms = t_ctc = t_ver = 0.0
                     ctc_b = ver_b = 0
+                    launches = 0.0
                     for sub in range(n_sub):
                         ws = synth.scaled(w, B=B // n_sub, seed=w.seed + 31 * sub)
                         sets = build_sets(ws, device, n_sets)
-                        a, b, c = time_steps(sets, steps, 5)
-                        ms, t_ctc, t_ver = ms + a, t_ctc + b, t_ver + c
-                        ctc_b += sets[0]["ctc_bytes"]
-                        ver_b += sets[0]["verify_bytes"]
+                        a, _, nl = timed_steps(sets, steps, 5)
+                        b, c, cb_, vb_ = time_kernels(sets)
+                        ms, t_ctc, t_ver = ms + a / steps, t_ctc + statistics.mean(b), t_ver + statistics.mean(c)
+                        launches += nl / steps
+                        ctc_b += cb_
+                        ver_b += vb_
                         del sets
                         torch.cuda.empty_cache()
                     nbytes = ctc_b + ver_b
                     line = {"point": w.name, "B": B, "V_llm": V, "dtype": dtype,
                             "sub_batches": n_sub, "input_sets": n_sets, "steps": steps,
-                            "logits_bytes": nbytes, "ms_per_step": round(ms, 5),
+                            "logits_bytes": int(nbytes), "ms_per_step": round(ms, 5),
+                            "gpu_launches_per_step": launches,
                             "utterances_per_s": round(B / (ms * 1e-3), 1),
                             "step_gbs": round(nbytes / (ms * 1e-3) / 1e9, 1),
                             "step_frac": round(nbytes / (ms * 1e-3) / 1e9 / peak, 4),
@@ -770,46 +895,25 @@ def run_stage1_only(args):
                       "dtype": w.dtype, "calls": 3}))
 
 
-def run_ring_sweep(args):
-    """ssd_verify's streaming kernel against the stage size of its ring (launch option
-    stage_bytes; 0 = the library's own choice): CUDA events the library records around the
-    kernel, rotating input sets, mean of 40 launches after 6 warm-up ones."""
+def run_verify_rows_only(args):
+    """ssd_verify alone on a few thousand rows of one configuration's LLM vocabulary (a GB or
+    two on the device), for a profiler capture of its kernels."""
     import torch
     from paper_2603_11243_b200 import binding as ssd
     from paper_2603_11243_b200 import build as lib_build
     from paper_2603_11243_b200 import synth
     lib_build.build()
     device = torch.device("cuda", 0)
-    torch.cuda.set_device(0)
-    w = synth.CONFIGS[args.config]
-    sets = build_sets(w, device, N_SETS)
-    code = ssd.BF16 if w.dtype == "bf16" else ssd.F32
-    row_bytes = w.V_llm * (2 if w.dtype == "bf16" else 4)
-    for sb in (0, 16512, 24704, 32896, 49280, 65536, 98432):
-        o = ssd.LaunchOpts()
-        o.stage_bytes = sb
-        try:
-            outs = [ssd.alloc_verify_outputs(s["M"], s["B"], device,
-                                             ssd.ssd_verify_workspace_bytes(s["B"], s["M"], w.V_llm, code, o))
-                    for s in sets]
-            n = 40
-            ev = make_events(2 * n)
-            for it in range(n + 6):
-                s = sets[it % len(sets)]
-                if it >= 6:
-                    o.ev_begin, o.ev_end = ev[2 * (it - 6)].cuda_event, ev[2 * (it - 6) + 1].cuda_event
-                ssd.ssd_verify(s["vb"].logits, s["tok_off"], s["ids"], w.tau_slm,
-                               skip=s["gate"]["gate_accept"], out=outs[it % len(sets)], opts=o)
-            torch.cuda.synchronize()
-        except ssd.SsdError as e:
-            print(json.dumps({"stage_bytes": sb, "refused": str(e)}), flush=True)
-            continue
-        us = statistics.mean(ev[2 * i].elapsed_time(ev[2 * i + 1]) for i in range(n)) * 1e3
-        nbytes = statistics.mean(s["verify_bytes"] for s in sets)
-        stages_per_row = None if sb == 0 else -(-(row_bytes + 32) // sb)
-        print(json.dumps({"workload": w.name, "stage_bytes": sb or "library default",
-                          "stages_per_row": stages_per_row, "kernel_us": round(us, 1),
-                          "gbs": round(nbytes / (us * 1e-6) / 1e9, 1)}), flush=True)
+    base = synth.CONFIGS[args.config]
+    per = min(base.max_draft_len, 200)
+    B = max(1, args.ncu_rows // per)
+    w = synth.scaled(base, B=B)
+    vb = synth.make_verify_batch(w, [per] * B, device)
+    for _ in range(3):
+        ssd.ssd_verify(vb.logits, vb.tok_off.to(device), vb.draft_ids.to(device), w.tau_slm)
+    torch.cuda.synchronize()
+    print(json.dumps({"verify_only": w.name, "rows": int(vb.logits.shape[0]), "V_llm": w.V_llm,
+                      "dtype": w.dtype, "calls": 3}))
 
 
 def main():
@@ -817,11 +921,11 @@ def main():
     if args.sweep:
         run_sweep(args)
         return
-    if args.ring_sweep:
-        run_ring_sweep(args)
-        return
     if args.ncu_stage1:
         run_stage1_only(args)
+        return
+    if args.ncu_rows:
+        run_verify_rows_only(args)
         return
     if args.impl == "reference":
         run_reference(args)

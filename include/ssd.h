@@ -78,6 +78,10 @@ typedef struct ssd_launch_opts {
                              polynomial on the FMA pipe instead of the special-function unit:
                              0 auto; 1..3 that many of the 4 pairs (ctc_draft: at most 2);
                              -1 none */
+    int32_t finish;       /* ssd_verify: where a row's log-likelihood and the utterance decisions
+                             are finished: 0 auto; 1 in a closing kernel of their own; 2 inside
+                             the streaming kernel (refused with SSD_ERR_ARG where that is not
+                             possible: column spans, the plain-load kernel, B > 2047) */
 } ssd_launch_opts;
 
 /* Human-readable name of a return code (static storage). */
@@ -88,6 +92,10 @@ int32_t ssd_last_cuda_error(void);
 
 /* Library version, major*10000 + minor*100 + patch. */
 int32_t ssd_version(void);
+
+/* Kernels this host thread has launched through the library so far (for launch accounting in
+ * benchmarks; the paper has no counterpart). */
+uint64_t ssd_launch_count(void);
 
 /* Bytes of device scratch the calls below need for these sizes and options (may be 0). */
 size_t ssd_ctc_draft_workspace_bytes(int32_t B, int64_t N, int32_t V, ssd_dtype dtype,
@@ -314,7 +322,8 @@ int32_t ssd_greedy_step(const void *logits, ssd_dtype dtype, int32_t V, int64_t 
  *
  * First call on a device: the function looks up the device address of the array (once per
  * device, under a lock, with the caller's current device).  Make that first call outside any
- * stream capture.  Later calls only read the cached address.
+ * stream capture.  Later calls only read the cached address.  `stream` must belong to the
+ * device that is current during the call: the array the kernels get is the current device's.
  *
  * Sharing: all calls on a device use the same array and it keeps whatever the last call left
  * in it.  Nothing in it needs clearing between calls.  Two calls whose kernels can run at the

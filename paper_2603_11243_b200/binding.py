@@ -33,7 +33,8 @@ class LaunchOpts(C.Structure):
     """Mirror of ssd_launch_opts (include/ssd.h)."""
     _fields_ = [("kernel", C.c_int32), ("ctas", C.c_int32), ("warps", C.c_int32),
                 ("stages", C.c_int32), ("stage_bytes", C.c_int32), ("split", C.c_int32),
-                ("ev_begin", C.c_void_p), ("ev_end", C.c_void_p), ("fma_exp", C.c_int32)]
+                ("ev_begin", C.c_void_p), ("ev_end", C.c_void_p), ("fma_exp", C.c_int32),
+                ("finish", C.c_int32)]
 
 
 _lib = None
@@ -51,6 +52,7 @@ def lib():
         L.ssd_status_string.argtypes = [C.c_int32]
         L.ssd_last_cuda_error.restype = C.c_int32
         L.ssd_version.restype = C.c_int32
+        L.ssd_launch_count.restype = C.c_uint64
         for f in (L.ssd_ctc_draft_workspace_bytes, L.ssd_verify_workspace_bytes):
             f.restype = C.c_size_t
             f.argtypes = [C.c_int32, C.c_int64, C.c_int32, C.c_int, C.c_void_p]

@@ -1,13 +1,67 @@
 // The C ABI of libssd: argument validation and dispatch.  Every step of the path runs in the
 // kernels of ssd_ctc.cu and ssd_verify.cu; nothing here computes.
+#include <map>
+#include <mutex>
+#include <utility>
+
 #include "ssd_common.cuh"
 
 namespace ssd {
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_mutex;
+int g_sm_count[kMaxDevices];                                   // 0: not asked yet
+std::map<std::pair<const void *, int>, size_t> g_smem_set;     // (kernel, device) -> bytes set
+thread_local int t_replay = 0;
+}  // namespace
+
+PlanReplay::PlanReplay() { ++t_replay; }
+PlanReplay::~PlanReplay() { --t_replay; }
+
+int device_sm_count() {
+    if (t_replay > 0) return 148;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (g_sm_count[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+            return 0;
+        g_sm_count[dev] = n;
+    }
+    return g_sm_count[dev];
+}
+
+cudaError_t ensure_dynamic_smem(const void *kernel, size_t bytes) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    size_t &have = g_smem_set[std::make_pair(kernel, dev)];
+    if (bytes <= have) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e == cudaSuccess) have = bytes;
+    return e;
+}
+
 static thread_local int32_t t_last_cuda_error = 0;
 void record_cuda_error(cudaError_t e) { t_last_cuda_error = (int32_t)e; }
+static thread_local uint64_t t_launches = 0;
+void count_launch() { ++t_launches; }
 }  // namespace ssd
 
 using namespace ssd;
+
+// The plan behind a call or a workspace query.  The shape of a launch depends on the device's
+// SM count; where no device can be asked (a host-only build step, an argument check without a
+// GPU) the plan is the one for the 148-SM part the kernels are tuned for, and a launch that
+// follows fails with SSD_ERR_CUDA.
+static int plan_for_query(int B, int64_t M, int V, ssd_dtype dtype, const ssd_launch_opts *opts,
+                          VerifyPlan *plan) {
+    if (device_sm_count() > 0) return plan_verify(B, M, V, dtype, opts, plan);
+    PlanReplay replay;
+    return plan_verify(B, M, V, dtype, opts, plan);
+}
 
 extern "C" {
 
@@ -28,7 +82,9 @@ const char *ssd_status_string(int32_t status) {
 
 int32_t ssd_last_cuda_error(void) { return t_last_cuda_error; }
 
-int32_t ssd_version(void) { return 100; }
+int32_t ssd_version(void) { return 200; }
+
+uint64_t ssd_launch_count(void) { return t_launches; }
 
 size_t ssd_ctc_draft_workspace_bytes(int32_t B, int64_t N, int32_t V, ssd_dtype dtype,
                                      const ssd_launch_opts *opts) {
@@ -42,7 +98,7 @@ size_t ssd_verify_workspace_bytes(int32_t B, int64_t M, int32_t V, ssd_dtype dty
                                   const ssd_launch_opts *opts) {
     if (B < 0 || M < 0 || V < 1 || (dtype != SSD_F32 && dtype != SSD_BF16)) return 0;
     VerifyPlan plan;
-    if (plan_verify(B, M, V, dtype, opts, &plan) != SSD_OK) return 0;
+    if (plan_for_query(B, M, V, dtype, opts, &plan) != SSD_OK) return 0;
     return plan.workspace_bytes;
 }
 
@@ -114,7 +170,7 @@ int32_t ssd_verify(const void *logits, ssd_dtype dtype, int32_t V, int64_t ld,
     const int es = dtype == SSD_F32 ? 4 : 2;
     if (reinterpret_cast<uintptr_t>(logits) % es) return SSD_ERR_ALIGN;
     VerifyPlan plan;
-    int rc = plan_verify(B, M, V, dtype, opts, &plan);
+    int rc = plan_for_query(B, M, V, dtype, opts, &plan);
     if (rc != SSD_OK) return rc;
     if (B > 0 && (!workspace || workspace_bytes < plan.workspace_bytes ||
                   reinterpret_cast<uintptr_t>(workspace) % 256))
@@ -136,7 +192,7 @@ int32_t ssd_verify_shard(const void *logits, ssd_dtype dtype, int32_t V_local, i
     const int es = dtype == SSD_F32 ? 4 : 2;
     if (reinterpret_cast<uintptr_t>(logits) % es) return SSD_ERR_ALIGN;
     VerifyPlan plan;
-    int rc = plan_verify(B, M, V_local, dtype, opts, &plan);
+    int rc = plan_for_query(B, M, V_local, dtype, opts, &plan);
     if (rc != SSD_OK) return rc;
     if (B > 0 && (!workspace || workspace_bytes < plan.workspace_bytes ||
                   reinterpret_cast<uintptr_t>(workspace) % 256))
@@ -196,7 +252,7 @@ size_t ssd_verify_early_exit_workspace_bytes(int32_t B, int64_t M, int32_t V, ss
                                              const ssd_launch_opts *opts) {
     if (B < 0 || M < 0 || V < 1 || (dtype != SSD_F32 && dtype != SSD_BF16)) return 0;
     VerifyPlan plan;
-    if (plan_verify(B, M, V, dtype, opts, &plan) != SSD_OK) return 0;
+    if (plan_for_query(B, M, V, dtype, opts, &plan) != SSD_OK) return 0;
     return verify_ee_workspace_bytes(B, plan);
 }
 
@@ -216,7 +272,7 @@ int32_t ssd_verify_early_exit(const void *logits, ssd_dtype dtype, int32_t V, in
     const int es = dtype == SSD_F32 ? 4 : 2;
     if (reinterpret_cast<uintptr_t>(logits) % es) return SSD_ERR_ALIGN;
     VerifyPlan plan;
-    int rc = plan_verify(B, M, V, dtype, opts, &plan);
+    int rc = plan_for_query(B, M, V, dtype, opts, &plan);
     if (rc != SSD_OK) return rc;
     if (B > 0 && (!workspace || workspace_bytes < verify_ee_workspace_bytes(B, plan) ||
                   reinterpret_cast<uintptr_t>(workspace) % 256))
@@ -242,7 +298,7 @@ size_t ssd_greedy_step_workspace_bytes(int64_t R, int32_t V, ssd_dtype dtype,
                                        const ssd_launch_opts *opts) {
     if (R < 0 || V < 1 || (dtype != SSD_F32 && dtype != SSD_BF16)) return 0;
     VerifyPlan plan;
-    if (plan_verify(0, R, V, dtype, opts, &plan) != SSD_OK) return 0;
+    if (plan_for_query(0, R, V, dtype, opts, &plan) != SSD_OK) return 0;
     return greedy_workspace_bytes(R, plan);
 }
 
@@ -256,7 +312,7 @@ int32_t ssd_greedy_step(const void *logits, ssd_dtype dtype, int32_t V, int64_t 
     const int es = dtype == SSD_F32 ? 4 : 2;
     if (reinterpret_cast<uintptr_t>(logits) % es) return SSD_ERR_ALIGN;
     VerifyPlan plan;
-    int rc = plan_verify(0, R, V, dtype, opts, &plan);
+    int rc = plan_for_query(0, R, V, dtype, opts, &plan);
     if (rc != SSD_OK) return rc;
     if (plan.kernel != 2) return SSD_ERR_ARG;
     if (R > 0 && (!workspace || workspace_bytes < greedy_workspace_bytes(R, plan) ||

@@ -39,6 +39,8 @@ __device__ __forceinline__ void pdl_enter() {
     pdl_wait();
 }
 
+void count_launch();     // one more kernel launched by this host thread (ssd_launch_count)
+
 template <typename... KArgs, typename... Args>
 cudaError_t launch_pdl(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem,
                        cudaStream_t stream, Args... args) {
@@ -52,6 +54,7 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), unsigned grid, unsigned block, 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    count_launch();
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
@@ -126,6 +129,62 @@ __device__ __forceinline__ void drain_after_error() {
     while (clock64() - t0 < (1ll << 22)) __nanosleep(1000);
 }
 
+// ---- scratch words that need no clearing ------------------------------------------------------
+// Adds k to a {epoch : 32 | count : 32} word and returns the count before the add.  A word
+// whose epoch is not this call's is a leftover (of an earlier call, or never written) and counts
+// as {epoch, 0}.  Epochs grow from call to call, so one atomic max with {epoch, 0} replaces a
+// leftover of an earlier call and leaves a word of this call alone; the add follows it without
+// waiting.  Only a leftover with a larger epoch field (memory that held something else) takes
+// the slow way: whoever sees it swaps {epoch, 0} in, and nobody adds before that has happened.
+__device__ __forceinline__ uint32_t tagged_finish(unsigned long long *w, uint32_t epoch, uint32_t k,
+                                                  unsigned long long old, bool &ok) {
+    if ((uint32_t)(old >> 32) == epoch) return (uint32_t)old;
+    const unsigned long long tag = (unsigned long long)epoch << 32;
+    for (int tries = 0; tries < (1 << 16); ++tries) {
+        const unsigned long long cur = *reinterpret_cast<volatile unsigned long long *>(w);
+        if ((uint32_t)(cur >> 32) == epoch) return (uint32_t)atomicAdd(w, (unsigned long long)k);
+        atomicCAS(w, cur, tag);
+    }
+    ok = false;
+    return 0xffffffffu;
+}
+__device__ __forceinline__ unsigned long long tagged_begin(unsigned long long *w, uint32_t epoch,
+                                                           uint32_t k) {
+    atomicMax(w, (unsigned long long)epoch << 32);
+    return atomicAdd(w, (unsigned long long)k);
+}
+__device__ __forceinline__ uint32_t tagged_add(unsigned long long *w, uint32_t epoch, uint32_t k,
+                                               bool &ok) {
+    return tagged_finish(w, epoch, k, tagged_begin(w, epoch, k), ok);
+}
+// Lowers a {epoch : 32 | value : 32} word to `value` (a leftover counts as "no value yet"), and
+// ORs bits into one (a leftover counts as 0).  Compare-and-swap loops: for updates that are rare.
+__device__ __forceinline__ void tagged_min(unsigned long long *w, uint32_t epoch, uint32_t value,
+                                           bool &ok) {
+    const unsigned long long mine = ((unsigned long long)epoch << 32) | value;
+    unsigned long long cur = *reinterpret_cast<volatile unsigned long long *>(w);
+    for (int tries = 0; tries < (1 << 12); ++tries) {
+        if ((uint32_t)(cur >> 32) == epoch && (uint32_t)cur <= value) return;
+        const unsigned long long old = atomicCAS(w, cur, mine);
+        if (old == cur) return;
+        cur = old;
+    }
+    ok = false;
+}
+__device__ __forceinline__ void tagged_or(unsigned long long *w, uint32_t epoch, uint32_t bits,
+                                          bool &ok) {
+    unsigned long long cur = *reinterpret_cast<volatile unsigned long long *>(w);
+    for (int tries = 0; tries < (1 << 12); ++tries) {
+        const uint32_t have = (uint32_t)(cur >> 32) == epoch ? (uint32_t)cur : 0u;
+        if ((uint32_t)(cur >> 32) == epoch && (have | bits) == have) return;
+        const unsigned long long old =
+            atomicCAS(w, cur, ((unsigned long long)epoch << 32) | have | bits);
+        if (old == cur) return;
+        cur = old;
+    }
+    ok = false;
+}
+
 // ---- arithmetic -------------------------------------------------------------------------------
 __device__ __forceinline__ float ex2(float x) {
     float y;
@@ -184,23 +243,6 @@ __device__ __forceinline__ float fmax_nan(float a, float b) {
     return d;
 }
 
-// (lo, hi) halves of a packed bf16 pair, each plus c, in fp32: the mixed-precision add of
-// sm_100 reads the 16-bit halves directly, so no unpacking instruction is needed.
-__device__ __forceinline__ float2 bf16x2_add_f32(uint32_t w, float c) {
-    float2 d;
-    asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\t"
-        "add.rn.f32.bf16 %0, lo, %3;\n\tadd.rn.f32.bf16 %1, hi, %3;\n\t}"
-        : "=f"(d.x), "=f"(d.y)
-        : "r"(w), "f"(c));
-    return d;
-}
-
-__device__ __forceinline__ float fmax_nan_fwd(float a, float b) {
-    float d;
-    asm("max.NaN.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
-    return d;
-}
-
 __device__ __forceinline__ float fmin_nan(float a, float b) {
     float d;
     asm("min.NaN.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
@@ -214,8 +256,8 @@ __device__ __forceinline__ float fmin_nan(float a, float b) {
 // exponent field would wrap), which the callers' range checks catch.  NaN passes the clamps.
 __device__ __forceinline__ float2 exp2_fma_pair(float2 t) {
     const float kMagic = 12582912.f;
-    t.x = fmin_nan(fmax_nan_fwd(t.x, -126.f), 128.f);
-    t.y = fmin_nan(fmax_nan_fwd(t.y, -126.f), 128.f);
+    t.x = fmin_nan(fmax_nan(t.x, -126.f), 128.f);
+    t.y = fmin_nan(fmax_nan(t.y, -126.f), 128.f);
     const float2 r = fadd2(t, make_float2(kMagic, kMagic));
     const float2 n = fadd2(r, make_float2(-kMagic, -kMagic));
     const float2 f = ffma2(n, make_float2(-1.f, -1.f), t);
@@ -357,7 +399,9 @@ struct VerifyPlan {
     int split;         // column spans per row
     int fma_exp;       // pairs per chunk whose exponential runs on the FMA pipe (bf16 only)
     int partials;      // partial (max, sum) pairs per row = split * warps
+    int finish_inside; // rows are finalised inside the streaming kernel (no closing kernel)
     size_t smem_bytes;
+    size_t fin_smem_bytes;
     size_t workspace_bytes;
 };
 int plan_verify(int B, int64_t M, int V, ssd_dtype dtype, const ssd_launch_opts *opts,
@@ -401,5 +445,18 @@ int launch_verify_ee(const void *logits, ssd_dtype dtype, int V, int64_t ld, int
                      int32_t *rows_read, const VerifyPlan &plan, const Launch &L);
 
 void record_cuda_error(cudaError_t e);
+
+// Multiprocessors of the current device (looked up once per device); <= 0 when the device cannot
+// be asked.  The host-only read-span hooks replay the plans without any device: while one of
+// them runs on this thread, the count of the part the kernels are tuned for (148) stands in.
+int device_sm_count();
+struct PlanReplay {
+    PlanReplay();
+    ~PlanReplay();
+};
+
+// cudaFuncAttributeMaxDynamicSharedMemorySize, set once per kernel and device (and again only
+// if a launch needs more than any before it).
+cudaError_t ensure_dynamic_smem(const void *kernel, size_t bytes);
 
 }  // namespace ssd

@@ -457,29 +457,6 @@ __device__ __forceinline__ MaxAt warp_max_at(MaxAt x) {
     return x;
 }
 
-// Adds k to a {epoch : 32 | count : 32} word and returns the count before the add.  A word
-// whose epoch is not this call's is a leftover (of an earlier call, or never written) and counts
-// as {epoch, 0}.  Epochs grow from call to call, so one atomic max with {epoch, 0} replaces a
-// leftover of an earlier call and leaves a word of this call alone; the add follows it without
-// waiting.  Only a leftover with a larger epoch field (memory that held something else) takes
-// the slow way: whoever sees it swaps {epoch, 0} in, and nobody adds before that has happened.
-__device__ __forceinline__ uint32_t tagged_finish(unsigned long long *w, uint32_t epoch, uint32_t k,
-                                                  unsigned long long old, bool &ok) {
-    if ((uint32_t)(old >> 32) == epoch) return (uint32_t)old;
-    const unsigned long long tag = (unsigned long long)epoch << 32;
-    for (int tries = 0; tries < (1 << 16); ++tries) {
-        const unsigned long long cur = *reinterpret_cast<volatile unsigned long long *>(w);
-        if ((uint32_t)(cur >> 32) == epoch) return (uint32_t)atomicAdd(w, (unsigned long long)k);
-        atomicCAS(w, cur, tag);
-    }
-    ok = false;
-    return 0xffffffffu;
-}
-__device__ __forceinline__ unsigned long long tagged_begin(unsigned long long *w, uint32_t epoch,
-                                                           uint32_t k) {
-    atomicMax(w, (unsigned long long)epoch << 32);
-    return atomicAdd(w, (unsigned long long)k);
-}
 // Shared memory: one mbarrier per warp | keep table | the warps' stages.
 //
 // Tiles: a warp's first tile is tile number (its index among all warps); further tiles are
@@ -825,21 +802,7 @@ __global__ void __launch_bounds__(256) gate_from_maxima_kernel(
     }
 }
 
-int g_sm_count = 0;
-int sm_count() {
-    if (g_sm_count == 0) {
-        int dev = 0, n = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-            n = 148;
-        g_sm_count = n;
-    }
-    return g_sm_count;
-}
-
 }  // namespace
-
-int device_sm_count() { return sm_count(); }
 
 unsigned long long next_epoch() {
     static unsigned long long counter = 0;
@@ -955,21 +918,24 @@ int launch_ctc_rows(const void *logits, ssd_dtype dtype, int V, int64_t ld, int6
         // small tiles are finished faster than a counter hands them out one by one
         p.claim = (int64_t)R * ld * es * p.counters < 3 * 12288 ? 2 : 1;
         int64_t ctas = (p.num_tiles + plan.warps - 1) / plan.warps;
-        const int max_ctas = (o && o->ctas > 0) ? o->ctas : sm_count();
+        const int sms = device_sm_count();
+        if (sms <= 0) { record_cuda_error(cudaErrorNoDevice); return SSD_ERR_CUDA; }
+        const int max_ctas = (o && o->ctas > 0) ? o->ctas : sms;
         if (ctas > max_ctas) ctas = max_ctas;
         void (*kern)(const CtcParams) = nullptr;
         if (dtype == SSD_F32) kern = pick_ctc<float, 0>(G);
         else kern = plan.fma_exp == 2 ? pick_ctc<bf16_t, 2>(G)
                   : plan.fma_exp == 1 ? pick_ctc<bf16_t, 1>(G) : pick_ctc<bf16_t, 0>(G);
-        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)plan.smem_bytes);
+        e = ensure_dynamic_smem(reinterpret_cast<const void *>(kern), plan.smem_bytes);
         if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
         e = launch_pdl(kern, (unsigned)ctas, (unsigned)(plan.warps * 32), plan.smem_bytes,
                        L.stream, p);
         if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
     } else {
         int64_t ctas = (N + 7) / 8;
-        const int64_t cap = (o && o->ctas > 0) ? o->ctas : (int64_t)sm_count() * 8;
+        const int sms = device_sm_count();
+        if (sms <= 0) { record_cuda_error(cudaErrorNoDevice); return SSD_ERR_CUDA; }
+        const int64_t cap = (o && o->ctas > 0) ? o->ctas : (int64_t)sms * 8;
         if (ctas > cap) ctas = cap;
         e = launch_pdl(dtype == SSD_F32 ? ctc_rows_plain<float> : ctc_rows_plain<bf16_t>,
                        (unsigned)ctas, 256u, 0, L.stream, p);

@@ -134,11 +134,14 @@ int launch_sweep(const float *utt_max_entropy, const float *token_logp, const in
             const double tau = (double)tau_slm[first + i];
             sp.tau_ctc[i] = tau_ctc[first + i];
             sp.reject_none[i] = !(tau > 0.0);
-            sp.log_tau_slm[i] = sp.reject_none[i] ? -INFINITY : (float)log(tau);
+            // tau >= 1 rejects everything (p <= 1), whatever rounding made of a stored log p
+            sp.log_tau_slm[i] = sp.reject_none[i] ? -INFINITY : tau >= 1.0 ? INFINITY : (float)log(tau);
         }
         const int64_t warps = (int64_t)sp.count * B;
         int64_t ctas = (warps + 7) / 8;
-        if (ctas > 148 * 8) ctas = 148 * 8;
+        const int sms = device_sm_count();
+        if (sms <= 0) return SSD_ERR_CUDA;
+        if (ctas > (int64_t)sms * 8) ctas = (int64_t)sms * 8;
         e = launch_pdl(sweep_kernel, (unsigned)ctas, 256u, 0, stream, utt_max_entropy, token_logp,
                        tok_off, B, M, sp, gate_accept, accepted_len, all_accepted, counts);
         if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }

@@ -30,6 +30,7 @@ int32_t ssd_ctc_draft_read_span(uint64_t base_addr, ssd_dtype dtype, int32_t V, 
     if (N < 0 || V < 1 || ld < V) return SSD_ERR_ARG;
     const int es = dtype == SSD_F32 ? 4 : 2;
     if (base_addr % es) return SSD_ERR_ALIGN;
+    PlanReplay replay;      // no device here: the plans use the SM count they are tuned for
     CtcPlan plan;
     const int rc = plan_ctc(dtype, V, ld, N, 0, opts, &plan);
     if (rc != SSD_OK) return rc;
@@ -92,6 +93,7 @@ int32_t ssd_verify_read_span(uint64_t base_addr, ssd_dtype dtype, int32_t V, int
     if (B < 0 || M < 0 || V < 1 || ld < V) return SSD_ERR_ARG;
     const int es = dtype == SSD_F32 ? 4 : 2;
     if (base_addr % es) return SSD_ERR_ALIGN;
+    PlanReplay replay;
     VerifyPlan plan;
     const int rc = plan_verify(B, M, V, dtype, opts, &plan);
     if (rc != SSD_OK) return rc;

@@ -27,7 +27,6 @@
 
 namespace ssd {
 
-int device_sm_count();
 
 namespace {
 
@@ -226,6 +225,353 @@ __global__ void __launch_bounds__(544, 1) verify_rows_tma(const VerifyParams p) 
     }
 }
 
+
+// Merge of a row's P (reference, sum) pairs into (maximum, sum relative to it).
+__device__ __forceinline__ float2 merge_partials(const float2 *pp, int P) {
+    float Mx = kNegInit, S = 0.f;
+    if ((P & 1) == 0 && P <= 16) {
+        const float4 *p4 = reinterpret_cast<const float4 *>(pp);
+        float4 v[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+            v[q] = q < P / 2 ? p4[q] : make_float4(kNegInit, 0.f, kNegInit, 0.f);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) Mx = fmaxf(Mx, fmaxf(v[q].x, v[q].z));
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+            S += v[q].y * ex2((v[q].x - Mx) * kLog2e) + v[q].w * ex2((v[q].z - Mx) * kLog2e);
+    } else {
+        for (int q = 0; q < P; ++q) Mx = fmaxf(Mx, pp[q].x);
+        for (int q = 0; q < P; ++q) {
+            const float2 v = pp[q];
+            S += v.y * ex2((v.x - Mx) * kLog2e);
+        }
+    }
+    return make_float2(Mx, S);
+}
+
+// Eq. 5 for one row, given its maximum Mx, ln of its sum of exponentials relative to Mx and the
+// draft token's logit x: the log-likelihood, whether the position is rejected (p <= tau; NaN
+// rejects; tau <= 0 rejects nothing, tau >= 1 everything), and the status bits the row raises.
+struct RowDecision {
+    float logp, lse;
+    bool reject;
+    uint32_t flags;
+};
+__device__ __forceinline__ RowDecision decide_row(float x, float Mx, float lnS, bool id_ok,
+                                                  float log_tau, int reject_none, int reject_all) {
+    RowDecision d;
+    d.lse = Mx + lnS;
+    d.flags = fabsf(d.lse) < INFINITY ? 0u : (uint32_t)SSD_UTT_NONFINITE;
+    if (!id_ok) {
+        d.flags |= SSD_UTT_BAD_DRAFT_ID;
+        d.logp = -INFINITY;
+        d.reject = true;
+    } else {
+        d.logp = (x - Mx) - lnS;      // not x - lse: keeps its accuracy when |x| is large
+        d.reject = reject_none ? false : (reject_all || !(d.logp > log_tau));
+    }
+    return d;
+}
+
+// ---- verification finished inside the streaming kernel ----------------------------------------
+// The same ring of stages as verify_rows_tma, for whole rows (no column spans).  The consumer
+// warps leave a row's (reference, sum) pairs in shared memory instead of the workspace; the
+// producer warp, when it next takes over the stage that held the row's last part and has the
+// stage's next copy under way, merges them, adds the draft token's logit (which it fetched,
+// with the draft id, one batch of rows ahead), writes the row's log-likelihood (Eq. 5) and, for
+// a rejected position, lowers the utterance's first-reject word in the workspace.  The CTA that
+// finishes last turns those words into accepted_len / all_accepted / utt_status (Section 2.3).
+// The words are {epoch : 32 | value : 32}: nothing has to be cleared between calls.
+struct FinParams {
+    VerifyParams v;
+    const int32_t *draft_ids;
+    float log_tau;
+    int reject_none, reject_all;
+    float *token_logp, *row_lse;
+    int32_t *accepted_len;
+    uint8_t *all_accepted;
+    uint32_t *utt_status;
+    unsigned long long *utt_words;     // [2 * B]: first rejected position, status bits
+    unsigned long long *done_ctas;
+    uint32_t epoch32;
+};
+
+struct FinRow {
+    int64_t row;
+    int32_t b, pos, id_ok;
+    float x;
+};
+
+__device__ __forceinline__ void utterance_outputs(int b, int64_t i0, int64_t i1, int64_t M,
+                                                  bool skipped, int first, uint32_t flags,
+                                                  uint32_t internal, int32_t *accepted_len,
+                                                  uint8_t *all_accepted, uint32_t *utt_status) {
+    if (i0 < 0 || i1 < i0 || i1 > M) {
+        accepted_len[b] = 0; all_accepted[b] = 0;
+        utt_status[b] = SSD_UTT_BAD_OFFSETS | internal;
+        return;
+    }
+    const int64_t K64 = i1 - i0;
+    const int K = K64 > 0x7fffffff ? 0x7fffffff : (int)K64;
+    if (skipped) { accepted_len[b] = K; all_accepted[b] = 1; utt_status[b] = internal; return; }
+    first = first < K ? first : K;
+    accepted_len[b] = first;
+    all_accepted[b] = first == K ? 1 : 0;
+    utt_status[b] = flags | internal;
+}
+
+template <typename T, int kF>
+__global__ void __launch_bounds__(544, 1) verify_rows_fin(const FinParams q) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    constexpr int ES = Elem<T>::kBytes, EPC = Elem<T>::kPerChunk;
+    __shared__ int s_last;
+    const VerifyParams &p = q.v;
+    pdl_launch_dependents();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int S = p.stages, CW = p.warps, NR = 2 * S;
+    // layout: full[S] | empty[S] | desc[S] | rows[NR] | spart[NR*CW] | pending[S] | offsets | stages
+    unsigned char *smem = reinterpret_cast<unsigned char *>(
+        (reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t full0 = sbase, empty0 = sbase + S * 8;
+    size_t o = 2 * (size_t)S * 8;
+    StageDesc *desc = reinterpret_cast<StageDesc *>(smem + o);     o += S * sizeof(StageDesc);
+    FinRow *rows = reinterpret_cast<FinRow *>(smem + o);           o += NR * sizeof(FinRow);
+    float2 *spart = reinterpret_cast<float2 *>(smem + o);          o += (size_t)NR * CW * 8;
+    int32_t *pending = reinterpret_cast<int32_t *>(smem + o);      o += S * 4;
+    o = (o + 7) & ~(size_t)7;
+    int64_t *offs = reinterpret_cast<int64_t *>(smem + o);         o += (size_t)(p.B + 1) * 8;
+    const uint32_t hdr = (uint32_t)((o + 127) & ~(size_t)127);
+    const uint32_t stage0 = sbase + hdr;
+    unsigned char *stage0_ptr = smem + hdr;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(full0 + s * 8, 1);
+            mbar_init(empty0 + s * 8, CW);
+            pending[s] = 0;
+        }
+        mbar_init_fence();
+        s_last = 0;
+    }
+    pdl_wait();
+    for (int i = threadIdx.x; i <= p.B; i += blockDim.x) offs[i] = p.tok_off[i];
+    __syncthreads();
+
+    const int64_t row_bytes = (int64_t)p.V * ES;
+    bool failed = false;
+
+    if (warp == 0) {
+        // =============================== producer ===============================
+        int s = 0;
+        uint32_t ph = 0;
+        int rowseq = 0;
+        bool ok = true;
+        const int max_chunks = p.stage_bytes >> 4;
+
+        auto finalize = [&](int slot1) {
+            if (slot1 == 0) return;
+            const int slot = slot1 - 1;
+            const float2 v = lane < CW ? spart[slot * CW + lane] : make_float2(kNegInit, 0.f);
+            const float Mx = fmaxf(warp_max(v.x), kNegInit);
+            const float Ssum = warp_sum(v.y * ex2((v.x - Mx) * kLog2e));
+            if (lane == 0) {
+                const FinRow rm = rows[slot];
+                const RowDecision d = decide_row(rm.x, Mx, logf(Ssum), rm.id_ok != 0, q.log_tau,
+                                                 q.reject_none, q.reject_all);
+                const float logp = d.logp, lse = d.lse;
+                const uint32_t fl = d.flags;
+                const bool reject = d.reject;
+                q.token_logp[rm.row] = logp;
+                if (q.row_lse) q.row_lse[rm.row] = lse;
+                if (fl) tagged_or(q.utt_words + 2 * rm.b + 1, q.epoch32, fl, ok);
+                if (reject) tagged_min(q.utt_words + 2 * rm.b, q.epoch32, (uint32_t)rm.pos, ok);
+            }
+            __syncwarp();
+        };
+
+        // What a lane knows about its row of a batch of 32 rows (row first + lane * grid): the
+        // utterance, the position, the draft id and the draft token's logit.  Loaded one batch
+        // ahead, so that nothing here waits for memory.
+        struct Mine { int64_t row; int b, pos, id; float x; bool active; };
+        auto look_up = [&](int64_t k0) {
+            Mine m{0, 0, 0, -1, 0.f, false};
+            m.row = (int64_t)blockIdx.x + (k0 + lane) * gridDim.x;
+            if (m.row < p.M) {
+                m.b = utterance_of_row(offs, p.B, m.row);
+                if (m.b >= 0) {
+                    const int64_t i0 = offs[m.b], i1 = offs[m.b + 1];
+                    m.active = i0 >= 0 && i1 <= p.M && m.row >= i0 && m.row < i1 &&
+                               i1 - i0 <= 0x7fffffff && !(p.skip && p.skip[m.b]);
+                    if (m.active) {
+                        m.pos = (int)(m.row - i0);
+                        m.id = q.draft_ids[m.row];
+                        if (m.id >= 0 && m.id < p.V)
+                            m.x = Elem<T>::load(p.logits + (m.row * p.ld + m.id) * ES);
+                    }
+                }
+            }
+            return m;
+        };
+        Mine next = look_up(0);
+        for (int64_t k0 = 0; !failed; k0 += 32) {
+            if ((int64_t)blockIdx.x + k0 * gridDim.x >= p.M) break;
+            const Mine cur = next;
+            next = look_up(k0 + 32);
+            unsigned todo = __ballot_sync(0xffffffffu, cur.active);
+            while (todo && !failed) {
+                const int src = __ffs(todo) - 1;
+                todo &= todo - 1;
+                const int64_t row = __shfl_sync(0xffffffffu, cur.row, src);
+                const int rslot = rowseq % NR;
+                ++rowseq;
+                if (lane == src) {
+                    FinRow rm;
+                    rm.row = cur.row; rm.b = cur.b; rm.pos = cur.pos;
+                    rm.id_ok = (cur.id >= 0 && cur.id < p.V) ? 1 : 0; rm.x = cur.x;
+                    rows[rslot] = rm;
+                }
+                const ranges::RowGeom geom = ranges::row_geom(
+                    reinterpret_cast<uintptr_t>(p.logits), row, p.ld * ES, row_bytes);
+                const uintptr_t g0 = geom.g0, g1 = geom.g1, f0 = geom.f0;
+                const ranges::SpanCut cut = ranges::span_cut(geom.row_chunks, 1, 0, max_chunks);
+                const int parts = cut.parts, per_part = cut.per_part;
+                for (int part = 0; part < parts; ++part) {
+                    if (!mbar_wait_bounded(empty0 + s * 8, ph ^ 1u)) { failed = true; break; }
+                    const int done_slot1 = pending[s];     // the row this stage held last, if any
+                    __syncwarp();
+                    const int pc0 = part * per_part;
+                    const int pc1 = min(geom.row_chunks, pc0 + per_part);
+                    const ranges::PartReads pr = ranges::part_reads(geom, pc0, pc1);
+                    const int b0 = pr.b0, b1 = pr.b1;
+                    unsigned char *dst = stage0_ptr + (size_t)s * p.stage_bytes;
+                    if (pr.head_plain) {
+                        if (lane < EPC) {
+                            const uintptr_t a = f0 + (uintptr_t)lane * ES;
+                            const bool in = a >= g0 && a < g1;
+                            if (ES == 4) reinterpret_cast<uint32_t *>(dst)[lane] =
+                                in ? *reinterpret_cast<const uint32_t *>(a) : 0xff800000u;
+                            else reinterpret_cast<uint16_t *>(dst)[lane] =
+                                in ? *reinterpret_cast<const uint16_t *>(a) : (uint16_t)0xff80u;
+                        }
+                    }
+                    if (pr.tail_plain) {
+                        if (lane < EPC) {
+                            const uintptr_t a = f0 + (uintptr_t)(pc1 - 1) * 16 + (uintptr_t)lane * ES;
+                            const bool in = a >= g0 && a < g1;
+                            unsigned char *d = dst + (size_t)(pc1 - 1 - pc0) * 16;
+                            if (ES == 4) reinterpret_cast<uint32_t *>(d)[lane] =
+                                in ? *reinterpret_cast<const uint32_t *>(a) : 0xff800000u;
+                            else reinterpret_cast<uint16_t *>(d)[lane] =
+                                in ? *reinterpret_cast<const uint16_t *>(a) : (uint16_t)0xff80u;
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) {
+                        const bool last = part == parts - 1;
+                        desc[s].nchunks = pc1 - pc0;
+                        desc[s].flags = last ? kFlagLast : 0u;
+                        desc[s].slot = rslot;
+                        desc[s].elem0 = 0;
+                        desc[s].gather = -1;
+                        pending[s] = last ? rslot + 1 : 0;
+                        const uint32_t bar = full0 + s * 8;
+                        if (b1 > b0) {
+                            const uint32_t bytes = (uint32_t)(b1 - b0) << 4;
+                            fence_proxy_async();
+                            mbar_arrive_expect_tx(bar, bytes);
+                            bulk_g2s(stage0 + (uint32_t)s * p.stage_bytes + ((uint32_t)(b0 - pc0) << 4),
+                                     reinterpret_cast<const void *>(f0 + ((uintptr_t)b0 << 4)),
+                                     bytes, bar);
+                        } else {
+                            mbar_arrive(bar);
+                        }
+                    }
+                    __syncwarp();
+                    finalize(done_slot1);     // after the stage's next copy is under way
+                    if (++s == S) { s = 0; ph ^= 1u; }
+                }
+            }
+        }
+        if (!failed) {
+            // end marker into the next stage, then the rows still waiting in the other stages
+            if (mbar_wait_bounded(empty0 + s * 8, ph ^ 1u)) {
+                finalize(pending[s]);
+                if (lane == 0) {
+                    desc[s].nchunks = 0; desc[s].flags = kFlagEnd; desc[s].slot = 0; desc[s].gather = -1;
+                    mbar_arrive(full0 + s * 8);
+                }
+                for (int t = 1; t < S && !failed; ++t) {
+                    const int st = (s + t) % S;
+                    const uint32_t par = st > s ? (ph ^ 1u) : ph;     // filled last round / this round
+                    if (mbar_wait_bounded(empty0 + st * 8, par)) finalize(pending[st]);
+                    else failed = true;
+                }
+            } else {
+                failed = true;
+            }
+        }
+        if (!__shfl_sync(0xffffffffu, (int)ok, 0)) failed = true;
+        if (failed) {
+            if (lane == 0) atomicExch(p.err_word, p.epoch);
+            drain_after_error();
+        }
+    } else {
+        // =============================== consumers ===============================
+        const int cw = warp - 1;
+        const int ct = cw * 32 + lane, NT = CW * 32;
+        Online st;
+        st.reset();
+        ArgTrack unused;
+        unused.reset();
+        int s = 0;
+        uint32_t ph = 0;
+        for (;;) {
+            if (!mbar_wait_bounded(full0 + s * 8, ph)) { failed = true; break; }
+            const int n = desc[s].nchunks;
+            const uint32_t flags = desc[s].flags;
+            if (flags & kFlagEnd) break;
+            consume_stage<T, kF, false>(stage0 + (uint32_t)s * p.stage_bytes, n, ct, NT, st, 0, unused);
+            if (flags & kFlagLast) {
+                const int slot = (int)desc[s].slot;
+                const float2 r = warp_merge(st);
+                if (lane == 0) spart[slot * CW + cw] = r;
+                st.reset();
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty0 + s * 8);      // releases the write above as well
+            if (++s == S) { s = 0; ph ^= 1u; }
+        }
+        if (failed) {
+            if (lane == 0) atomicExch(p.err_word, p.epoch);
+            drain_after_error();
+        }
+    }
+
+    // ---- the CTA that finishes last writes the per-utterance outputs --------------------------
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        bool ok2 = true;
+        const uint32_t before = tagged_add(q.done_ctas, q.epoch32, 1u, ok2);
+        s_last = ok2 && before + 1 == gridDim.x;
+        if (!ok2) atomicExch(p.err_word, p.epoch);
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    const uint32_t internal = (__ldcg(p.err_word) == p.epoch) ? (uint32_t)SSD_UTT_INTERNAL : 0u;
+    for (int b = threadIdx.x; b < p.B; b += blockDim.x) {
+        const unsigned long long w0 = __ldcg(q.utt_words + 2 * b), w1 = __ldcg(q.utt_words + 2 * b + 1);
+        const int first = (uint32_t)(w0 >> 32) == q.epoch32 ? (int)min((uint32_t)w0, 0x7fffffffu)
+                                                            : 0x7fffffff;
+        const uint32_t fl = (uint32_t)(w1 >> 32) == q.epoch32 ? (uint32_t)w1 : 0u;
+        utterance_outputs(b, offs[b], offs[b + 1], p.M, p.skip && p.skip[b], first, fl, internal,
+                          q.accepted_len, q.all_accepted, q.utt_status);
+    }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(256) verify_rows_plain(const VerifyParams p) {
     constexpr int ES = Elem<T>::kBytes;
@@ -260,7 +606,7 @@ template <typename T>
 __global__ void __launch_bounds__(kFinishThreads) verify_finish_kernel(
     const char *__restrict__ logits, int V, int64_t ld, int64_t M,
     const int64_t *__restrict__ tok_off, const int32_t *__restrict__ draft_ids, int B,
-    float log_tau, int reject_none, const uint8_t *__restrict__ skip,
+    float log_tau, int reject_none, int reject_all, const uint8_t *__restrict__ skip,
     const float2 *__restrict__ partials, int P, float *__restrict__ token_logp,
     float *__restrict__ row_lse, int32_t *__restrict__ accepted_len,
     uint8_t *__restrict__ all_accepted, uint32_t *__restrict__ utt_status,
@@ -298,45 +644,15 @@ __global__ void __launch_bounds__(kFinishThreads) verify_finish_kernel(
         const int64_t r = i0 + i;
         const int id = draft_ids[r];
         const bool id_ok = id >= 0 && id < V;
-        // P (reference, sum) pairs of this row; up to 16 are read two at a time into registers
-        const float2 *pp = partials + r * P;
-        float Mx = kNegInit, S = 0.f;
+        // the row's partials and the draft token's logit are fetched together
         float x = 0.f;
-        if ((P & 1) == 0 && P <= 16) {
-            const float4 *p4 = reinterpret_cast<const float4 *>(pp);
-            float4 v[8];
-#pragma unroll
-            for (int q = 0; q < 8; ++q)
-                v[q] = q < P / 2 ? p4[q] : make_float4(kNegInit, 0.f, kNegInit, 0.f);
-            if (id_ok) x = Elem<T>::load(logits + (r * ld + id) * ES);
-#pragma unroll
-            for (int q = 0; q < 8; ++q) Mx = fmaxf(Mx, fmaxf(v[q].x, v[q].z));
-#pragma unroll
-            for (int q = 0; q < 8; ++q)
-                S += v[q].y * ex2((v[q].x - Mx) * kLog2e) + v[q].w * ex2((v[q].z - Mx) * kLog2e);
-        } else {
-            if (id_ok) x = Elem<T>::load(logits + (r * ld + id) * ES);
-            for (int q = 0; q < P; ++q) Mx = fmaxf(Mx, pp[q].x);
-            for (int q = 0; q < P; ++q) {
-                const float2 v = pp[q];
-                S += v.y * ex2((v.x - Mx) * kLog2e);
-            }
-        }
-        const float lnS = logf(S);
-        const float lse = Mx + lnS;
-        if (!(fabsf(lse) < INFINITY)) myflags |= SSD_UTT_NONFINITE;
-        float logp;
-        bool reject;
-        if (!id_ok) {
-            myflags |= SSD_UTT_BAD_DRAFT_ID;
-            logp = -INFINITY;
-            reject = true;
-        } else {
-            logp = (x - Mx) - lnS;      // not x - lse: keeps its accuracy when |x| is large
-            reject = reject_none ? false : !(logp > log_tau);   // p <= tau; NaN rejects
-        }
-        token_logp[r] = logp;
-        if (row_lse) row_lse[r] = lse;
+        if (id_ok) x = Elem<T>::load(logits + (r * ld + id) * ES);
+        const float2 ms = merge_partials(partials + r * P, P);
+        const RowDecision d = decide_row(x, ms.x, logf(ms.y), id_ok, log_tau, reject_none, reject_all);
+        myflags |= d.flags;
+        token_logp[r] = d.logp;
+        if (row_lse) row_lse[r] = d.lse;
+        const bool reject = d.reject;
         if (reject && i < myfirst) myfirst = i;
     }
     if (myfirst < K) atomicMin(&first_reject, myfirst);
@@ -347,30 +663,6 @@ __global__ void __launch_bounds__(kFinishThreads) verify_finish_kernel(
         all_accepted[b] = first_reject == K ? 1 : 0;
         utt_status[b] = flags | internal;
     }
-}
-
-// Merge of a row's P (reference, sum) pairs into (maximum, sum relative to it).
-__device__ __forceinline__ float2 merge_partials(const float2 *pp, int P) {
-    float Mx = kNegInit, S = 0.f;
-    if ((P & 1) == 0 && P <= 16) {
-        const float4 *p4 = reinterpret_cast<const float4 *>(pp);
-        float4 v[8];
-#pragma unroll
-        for (int q = 0; q < 8; ++q)
-            v[q] = q < P / 2 ? p4[q] : make_float4(kNegInit, 0.f, kNegInit, 0.f);
-#pragma unroll
-        for (int q = 0; q < 8; ++q) Mx = fmaxf(Mx, fmaxf(v[q].x, v[q].z));
-#pragma unroll
-        for (int q = 0; q < 8; ++q)
-            S += v[q].y * ex2((v[q].x - Mx) * kLog2e) + v[q].w * ex2((v[q].z - Mx) * kLog2e);
-    } else {
-        for (int q = 0; q < P; ++q) Mx = fmaxf(Mx, pp[q].x);
-        for (int q = 0; q < P; ++q) {
-            const float2 v = pp[q];
-            S += v.y * ex2((v.x - Mx) * kLog2e);
-        }
-    }
-    return make_float2(Mx, S);
 }
 
 constexpr uint32_t kStatsInternal = 0x7fc0dead;   // in place of a row's maximum: a wait ran out
@@ -412,7 +704,7 @@ __global__ void __launch_bounds__(kFinishThreads) shard_finish_kernel(
 __global__ void __launch_bounds__(kFinishThreads) combine_kernel(
     const float *__restrict__ stats_all, int R, int64_t V_total, int64_t M,
     const int64_t *__restrict__ tok_off, const int32_t *__restrict__ draft_ids, int B,
-    float log_tau, int reject_none, const uint8_t *__restrict__ skip,
+    float log_tau, int reject_none, int reject_all, const uint8_t *__restrict__ skip,
     float *__restrict__ token_logp, float *__restrict__ row_lse,
     int32_t *__restrict__ accepted_len, uint8_t *__restrict__ all_accepted,
     uint32_t *__restrict__ utt_status) {
@@ -453,21 +745,11 @@ __global__ void __launch_bounds__(kFinishThreads) combine_kernel(
             const float *t = stats_all + ((int64_t)q * M + r) * 3;
             S += t[1] * ex2((t[0] - Mx) * kLog2e);
         }
-        const float lnS = logf(S);
-        const float lse = Mx + lnS;
-        if (!(fabsf(lse) < INFINITY)) myflags |= SSD_UTT_NONFINITE;
-        float logp;
-        bool reject;
-        if (!id_ok) {
-            myflags |= SSD_UTT_BAD_DRAFT_ID;
-            logp = -INFINITY;
-            reject = true;
-        } else {
-            logp = (x - Mx) - lnS;
-            reject = reject_none ? false : !(logp > log_tau);
-        }
-        token_logp[r] = logp;
-        if (row_lse) row_lse[r] = lse;
+        const RowDecision d = decide_row(x, Mx, logf(S), id_ok, log_tau, reject_none, reject_all);
+        myflags |= d.flags;
+        token_logp[r] = d.logp;
+        if (row_lse) row_lse[r] = d.lse;
+        const bool reject = d.reject;
         if (reject && i < myfirst) myfirst = i;
     }
     if (myfirst < K) atomicMin(&first_reject, myfirst);
@@ -525,7 +807,8 @@ __global__ void __launch_bounds__(kGreedyWarps * 32) greedy_finish_kernel(
 
 unsigned long long next_epoch();
 
-// Workspace: [0,256) header (error word), then M * partials float2.
+// Workspace: [0,256) header (error word, finished-CTA counter), two words per utterance, then
+// M * partials float2.
 int plan_verify(int B, int64_t M, int V, ssd_dtype dtype, const ssd_launch_opts *o,
                 VerifyPlan *plan) {
     const int es = dtype == SSD_F32 ? 4 : 2;
@@ -533,6 +816,7 @@ int plan_verify(int B, int64_t M, int V, ssd_dtype dtype, const ssd_launch_opts 
     pl.kernel = (o && o->kernel) ? o->kernel : 2;
     if (pl.kernel != 1 && pl.kernel != 2) return SSD_ERR_ARG;
     const int sms = device_sm_count();
+    if (sms <= 0 && !(o && o->ctas > 0)) return SSD_ERR_CUDA;
     pl.ctas = (o && o->ctas > 0) ? o->ctas : sms;
     const int64_t row_bytes = (int64_t)V * es;
     // column spans per row: enough items for a few balanced waves when there are few rows
@@ -588,9 +872,28 @@ int plan_verify(int B, int64_t M, int V, ssd_dtype dtype, const ssd_launch_opts 
     pl.fma_exp = (o && o->fma_exp) ? (o->fma_exp < 0 ? 0 : o->fma_exp) : (dtype == SSD_BF16 ? 1 : 0);
     if (pl.fma_exp > 3) return SSD_ERR_ARG;
     pl.partials = split * pl.warps;
-    pl.workspace_bytes = 256 + (size_t)M * pl.partials * sizeof(float2);
+    // header | two words per utterance | partials
+    pl.workspace_bytes = 256 + (((size_t)(B > 0 ? B : 0) * 16 + 255) & ~(size_t)255) +
+                         (size_t)M * pl.partials * sizeof(float2);
+    // rows are finished inside the streaming kernel where that kernel sees whole rows and can
+    // keep the utterance offsets in shared memory
+    const int finish = o ? o->finish : 0;
+    if (finish < 0 || finish > 2) return SSD_ERR_ARG;
+    pl.finish_inside = 0;
+    if (finish != 1 && pl.kernel == 2 && split == 1 && B > 0 && B + 1 <= kOffCacheMax && M > 0) {
+        const int NR = 2 * pl.stages;
+        size_t hdr = 2 * (size_t)pl.stages * 8 + pl.stages * sizeof(StageDesc) + NR * sizeof(FinRow) +
+                     (size_t)NR * pl.warps * 8 + pl.stages * 4 + 8 + (size_t)(B + 1) * 8;
+        pl.fin_smem_bytes = 128 + ((hdr + 127) & ~(size_t)127) + (size_t)pl.stages * pl.stage_bytes;
+        pl.finish_inside = pl.fin_smem_bytes <= 227 * 1024 ? 1 : 0;
+    }
+    if (finish == 2 && !pl.finish_inside) return SSD_ERR_ARG;
     *plan = pl;
     return SSD_OK;
+}
+
+static size_t partials_offset(int B) {
+    return 256 + (((size_t)(B > 0 ? B : 0) * 16 + 255) & ~(size_t)255);
 }
 
 // Launches the streaming kernel that leaves plan.partials (reference, sum) pairs per row in the
@@ -605,7 +908,7 @@ static int launch_verify_rows(const void *logits, ssd_dtype dtype, int V, int64_
     p.logits = static_cast<const char *>(logits);
     p.V = V; p.ld = ld; p.M = M; p.split = plan.split; p.num_items = M * plan.split;
     p.tok_off = tok_off; p.B = B; p.skip = skip;
-    p.partials = reinterpret_cast<float2 *>(static_cast<char *>(workspace) + 256);
+    p.partials = reinterpret_cast<float2 *>(static_cast<char *>(workspace) + partials_offset(B));
     p.partials_per_row = plan.partials;
     p.warps = plan.warps; p.stages = plan.stages; p.stage_bytes = plan.stage_bytes;
     p.err_word = static_cast<unsigned long long *>(workspace); p.epoch = epoch;
@@ -621,8 +924,7 @@ static int launch_verify_rows(const void *logits, ssd_dtype dtype, int V, int64_
                  : plan.fma_exp == 2 ? verify_rows_tma<bf16_t, 2, false>
                  : plan.fma_exp == 3 ? verify_rows_tma<bf16_t, 3, false>
                                      : verify_rows_tma<bf16_t, 0, false>;
-        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)plan.smem_bytes);
+        e = ensure_dynamic_smem(reinterpret_cast<const void *>(kern), plan.smem_bytes);
         if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
         e = launch_pdl(kern, (unsigned)ctas, (unsigned)((plan.warps + 1) * 32), plan.smem_bytes,
                        L.stream, p);
@@ -642,26 +944,79 @@ static int launch_verify_rows(const void *logits, ssd_dtype dtype, int V, int64_
     return SSD_OK;
 }
 
+// Eq. 5's threshold on the host: log(tau) in fp64, rounded to fp32.  tau <= 0 rejects nothing
+// (p > 0 always), tau >= 1 everything (p <= 1 always), whatever rounding does to log p.
+struct Threshold {
+    float log_tau;
+    int reject_none, reject_all;
+};
+static Threshold threshold_of(float tau_slm) {
+    const double tau = (double)tau_slm;
+    Threshold t;
+    t.reject_none = !(tau > 0.0);
+    t.reject_all = tau >= 1.0;
+    t.log_tau = t.reject_none ? -INFINITY : (float)log(tau);
+    return t;
+}
+
 int launch_verify(const void *logits, ssd_dtype dtype, int V, int64_t ld, int64_t M,
                   const int64_t *tok_off, const int32_t *draft_ids, int B, float tau_slm,
                   const uint8_t *skip, void *workspace, float *token_logp, float *row_lse,
                   int32_t *accepted_len, uint8_t *all_accepted, uint32_t *utt_status,
                   const VerifyPlan &plan, const Launch &L) {
     if (B == 0) return SSD_OK;
+    const ssd_launch_opts *o = L.opts;
     unsigned long long *err_word = static_cast<unsigned long long *>(workspace);
-    float2 *partials = reinterpret_cast<float2 *>(static_cast<char *>(workspace) + 256);
+    float2 *partials = reinterpret_cast<float2 *>(static_cast<char *>(workspace) + partials_offset(B));
     const unsigned long long epoch = next_epoch();
+    const Threshold th = threshold_of(tau_slm);
+    cudaError_t e;
+    if (plan.finish_inside) {
+        FinParams q{};
+        VerifyParams &p = q.v;
+        p.logits = static_cast<const char *>(logits);
+        p.V = V; p.ld = ld; p.M = M; p.split = 1; p.num_items = M;
+        p.tok_off = tok_off; p.B = B; p.skip = skip;
+        p.warps = plan.warps; p.stages = plan.stages; p.stage_bytes = plan.stage_bytes;
+        p.err_word = err_word; p.epoch = epoch;
+        q.draft_ids = draft_ids;
+        q.log_tau = th.log_tau; q.reject_none = th.reject_none; q.reject_all = th.reject_all;
+        q.token_logp = token_logp; q.row_lse = row_lse;
+        q.accepted_len = accepted_len; q.all_accepted = all_accepted; q.utt_status = utt_status;
+        q.utt_words = reinterpret_cast<unsigned long long *>(static_cast<char *>(workspace) + 256);
+        q.done_ctas = err_word + 1;
+        q.epoch32 = (uint32_t)epoch;
+        const int64_t ctas = M < plan.ctas ? M : plan.ctas;
+        if (o && o->ev_begin) {
+            e = cudaEventRecord(static_cast<cudaEvent_t>(o->ev_begin), L.stream);
+            if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
+        }
+        void (*kern)(const FinParams) = verify_rows_fin<float, 0>;
+        if (dtype == SSD_BF16)
+            kern = plan.fma_exp == 1 ? verify_rows_fin<bf16_t, 1>
+                 : plan.fma_exp == 2 ? verify_rows_fin<bf16_t, 2>
+                 : plan.fma_exp == 3 ? verify_rows_fin<bf16_t, 3>
+                                     : verify_rows_fin<bf16_t, 0>;
+        e = ensure_dynamic_smem(reinterpret_cast<const void *>(kern), plan.fin_smem_bytes);
+        if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
+        e = launch_pdl(kern, (unsigned)ctas, (unsigned)((plan.warps + 1) * 32), plan.fin_smem_bytes,
+                       L.stream, q);
+        if (e == cudaSuccess) e = cudaGetLastError();
+        if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
+        if (o && o->ev_end) {
+            e = cudaEventRecord(static_cast<cudaEvent_t>(o->ev_end), L.stream);
+            if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
+        }
+        return SSD_OK;
+    }
     const int rc = launch_verify_rows(logits, dtype, V, ld, M, tok_off, B, skip, workspace, epoch,
                                       plan, L);
     if (rc != SSD_OK) return rc;
-    const double tau = (double)tau_slm;
-    const int reject_none = !(tau > 0.0);
-    const float log_tau = reject_none ? -INFINITY : (float)log(tau);
-    cudaError_t e = launch_pdl(
+    e = launch_pdl(
         dtype == SSD_F32 ? verify_finish_kernel<float> : verify_finish_kernel<bf16_t>,
         (unsigned)B, (unsigned)kFinishThreads, 0, L.stream,
-        static_cast<const char *>(logits), V, ld, M, tok_off, draft_ids, B, log_tau,
-        reject_none, skip, static_cast<const float2 *>(partials), plan.partials,
+        static_cast<const char *>(logits), V, ld, M, tok_off, draft_ids, B, th.log_tau,
+        th.reject_none, th.reject_all, skip, static_cast<const float2 *>(partials), plan.partials,
         token_logp, row_lse, accepted_len, all_accepted, utt_status,
         static_cast<const unsigned long long *>(err_word), epoch);
     if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
@@ -678,7 +1033,7 @@ int launch_verify_shard(const void *logits, ssd_dtype dtype, int V_local, int64_
                         const VerifyPlan &plan, const Launch &L) {
     if (B == 0) return SSD_OK;
     unsigned long long *err_word = static_cast<unsigned long long *>(workspace);
-    float2 *partials = reinterpret_cast<float2 *>(static_cast<char *>(workspace) + 256);
+    float2 *partials = reinterpret_cast<float2 *>(static_cast<char *>(workspace) + partials_offset(B));
     const unsigned long long epoch = next_epoch();
     const int rc = launch_verify_rows(logits, dtype, V_local, ld, M, tok_off, B, skip, workspace,
                                       epoch, plan, L);
@@ -701,13 +1056,11 @@ int launch_verify_combine(const float *stats_all, int R, int64_t V_total, const 
                           int32_t *accepted_len, uint8_t *all_accepted, uint32_t *utt_status,
                           cudaStream_t stream) {
     if (B == 0) return SSD_OK;
-    const double tau = (double)tau_slm;
-    const int reject_none = !(tau > 0.0);
-    const float log_tau = reject_none ? -INFINITY : (float)log(tau);
+    const Threshold th = threshold_of(tau_slm);
     cudaError_t e = launch_pdl(combine_kernel, (unsigned)B, (unsigned)kFinishThreads, 0, stream,
-                               stats_all, R, V_total, M, tok_off, draft_ids, B, log_tau,
-                               reject_none, skip, token_logp, row_lse, accepted_len, all_accepted,
-                               utt_status);
+                               stats_all, R, V_total, M, tok_off, draft_ids, B, th.log_tau,
+                               th.reject_none, th.reject_all, skip, token_logp, row_lse,
+                               accepted_len, all_accepted, utt_status);
     if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
     e = cudaGetLastError();
     if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
@@ -743,7 +1096,7 @@ int launch_greedy(const void *logits, ssd_dtype dtype, int V, int64_t ld, int64_
     void (*kern)(const VerifyParams) = verify_rows_tma<float, 0, true>;
     if (dtype == SSD_BF16)
         kern = plan.fma_exp >= 1 ? verify_rows_tma<bf16_t, 1, true> : verify_rows_tma<bf16_t, 0, true>;
-    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
+    e = ensure_dynamic_smem(reinterpret_cast<const void *>(kern), plan.smem_bytes);
     if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
     e = launch_pdl(kern, (unsigned)ctas, (unsigned)((plan.warps + 1) * 32), plan.smem_bytes,
                    L.stream, p);

@@ -22,7 +22,6 @@
 
 namespace ssd {
 
-int device_sm_count();
 unsigned long long next_epoch();
 
 namespace {
@@ -39,7 +38,7 @@ struct EeParams {
     int B;
     const uint8_t *skip;
     float log_tau;
-    int reject_none;
+    int reject_none, reject_all;
     float *token_logp;
     float *row_lse;
     int32_t *first_reject;     // [B] lowest rejected position known so far (K_b: none)
@@ -161,7 +160,7 @@ __global__ void __launch_bounds__(544, 1) verify_rows_ee(const EeParams p) {
                     reject = true;
                 } else {
                     logp = (sx[slot] - Mx) - lnS;
-                    reject = p.reject_none ? false : !(logp > p.log_tau);   // p <= tau; NaN rejects
+                    reject = p.reject_none ? false : (p.reject_all || !(logp > p.log_tau));   // p <= tau; NaN rejects
                 }
                 p.token_logp[rm.row] = logp;
                 if (p.row_lse) p.row_lse[rm.row] = lse;
@@ -424,6 +423,7 @@ int launch_verify_ee(const void *logits, ssd_dtype dtype, int V, int64_t ld, int
     p.skip = skip;
     const double tau = (double)tau_slm;
     p.reject_none = !(tau > 0.0);
+    p.reject_all = tau >= 1.0;     // p <= 1 always, whatever rounding makes of log p
     p.log_tau = p.reject_none ? -INFINITY : (float)log(tau);
     p.token_logp = token_logp; p.row_lse = row_lse;
     p.first_reject = first_reject; p.flags = flags; p.rows_read = rr; p.kmax = kmax;
@@ -441,7 +441,7 @@ int launch_verify_ee(const void *logits, ssd_dtype dtype, int V, int64_t ld, int
     }
     void (*kern)(const EeParams) = verify_rows_ee<float, 0>;
     if (dtype == SSD_BF16) kern = plan.fma_exp >= 1 ? verify_rows_ee<bf16_t, 1> : verify_rows_ee<bf16_t, 0>;
-    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    e = ensure_dynamic_smem(reinterpret_cast<const void *>(kern), smem);
     if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
     e = launch_pdl(kern, (unsigned)plan.ctas, (unsigned)((plan.warps + 1) * 32), smem, L.stream, p);
     if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }

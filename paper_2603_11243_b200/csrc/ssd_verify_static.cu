@@ -56,7 +56,11 @@ extern "C" int32_t ssd_verify_static(const void *logits, ssd_dtype dtype, int32_
     if (dtype != SSD_F32 && dtype != SSD_BF16) return SSD_ERR_DTYPE;
     if (B < 0 || M < 0 || V < 1 || ld < V) return SSD_ERR_ARG;
     VerifyPlan plan;
-    int rc = plan_verify(B, M, V, dtype, opts, &plan);
+    int rc = device_sm_count() > 0 ? plan_verify(B, M, V, dtype, opts, &plan) : SSD_ERR_CUDA;
+    if (rc == SSD_ERR_CUDA) {              // no device to ask: the size check still works
+        PlanReplay replay;
+        rc = plan_verify(B, M, V, dtype, opts, &plan);
+    }
     if (rc != SSD_OK) return rc;
     if (plan.workspace_bytes > kStaticScratchBytes) return SSD_ERR_TOO_LARGE;
     void *scratch = nullptr;

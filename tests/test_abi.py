@@ -121,7 +121,8 @@ def test_workspace_queries(lib):
     assert small >= 256 + 250 * 8 * 8 and big >= 256 + 6400 * 8 * 8
     o = ssd.LaunchOpts()
     o.split, o.warps = 4, 8
-    assert ssd.ssd_verify_workspace_bytes(32, 6400, 49152, ssd.BF16, o) == 256 + 6400 * 4 * 8 * 8
+    # header, two words per utterance (rounded to 256 bytes), 8-byte pairs per row, span and warp
+    assert ssd.ssd_verify_workspace_bytes(32, 6400, 49152, ssd.BF16, o) == 256 + 512 + 6400 * 4 * 8 * 8
 
 
 def test_binding_refuses_host_tensors(lib):

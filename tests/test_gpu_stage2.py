@@ -10,7 +10,16 @@ from paper_2603_11243_b200 import synth
 
 pytestmark = pytest.mark.gpu
 
-KERNELS = {"plain": 1, "tma": 2}
+# plain loads; bulk copies with rows finished inside the streaming kernel; bulk copies with the
+# closing kernel of its own
+KERNELS = {"plain": dict(kernel=1), "tma": dict(kernel=2, finish=2, split=1),
+           "tma_closing": dict(kernel=2, finish=1)}
+
+
+def _kopts(kernel, okw):
+    k = dict(kernel) if isinstance(kernel, dict) else {"kernel": kernel}
+    k.update(okw)
+    return k
 
 
 def run_verify(logits_dev, tok_off, draft_ids, V, tau, skip=None, guard=True, **okw):
@@ -36,7 +45,7 @@ def run_verify(logits_dev, tok_off, draft_ids, V, tau, skip=None, guard=True, **
 def check_verify(w, K, device, kernel, skip=None, require_all_margins=True, **okw):
     vb = synth.make_verify_batch(w, K, "cpu")
     out = run_verify(vb.logits.to(device), vb.tok_off, vb.draft_ids, w.V_llm, w.tau_slm,
-                     skip=skip, kernel=kernel, **okw)
+                     skip=skip, **_kopts(kernel, okw))
     orc = ref.verify(H.storage_numpy(vb.logits), w.V_llm, vb.tok_off.numpy(),
                      vb.draft_ids.numpy(), float(np.float32(w.tau_slm)), skip=skip)
     H.compare_stage2(out, orc, vb.tok_off.numpy(), w.tau_slm, skip=skip,
@@ -114,7 +123,7 @@ def test_padded_rows_and_misaligned_base(cuda_device, kernel, dtype):
     vb = synth.make_verify_batch(w, [6, 1, 9], "cpu")
     ids = (vb.draft_ids % V).to(torch.int32)
     wide = vb.logits.to(cuda_device)
-    out = run_verify(wide[:, 5:5 + V], vb.tok_off, ids, V, 0.1, kernel=kernel)
+    out = run_verify(wide[:, 5:5 + V], vb.tok_off, ids, V, 0.1, **kernel)
     orc = ref.verify(H.storage_numpy(vb.logits[:, 5:5 + V].contiguous()), V, vb.tok_off.numpy(),
                      ids.numpy(), float(np.float32(0.1)))
     H.compare_stage2(out, orc, vb.tok_off.numpy(), 0.1, require_all_margins=False)
@@ -135,7 +144,7 @@ def test_bad_draft_ids_nonfinite_rows_and_thresholds(cuda_device, kernel):
     x2 = x.clone()
     x2[0, 3] = float("nan")   # utterance 0, row 0
     x2[2, :10] = -float("inf")  # masked entries are fine
-    out = run_verify(x2.to(cuda_device), off, bad, V, 0.1, kernel=kernel)
+    out = run_verify(x2.to(cuda_device), off, bad, V, 0.1, **kernel)
     st = H.status_u32(out["utt_status"])
     assert st[0] == ssd.UTT_NONFINITE and st[1] == ssd.UTT_BAD_DRAFT_ID and st[2] == ssd.UTT_BAD_DRAFT_ID
     assert list(out["accepted_len"].cpu().numpy()) == [0, 1, 1]
@@ -143,10 +152,18 @@ def test_bad_draft_ids_nonfinite_rows_and_thresholds(cuda_device, kernel):
     np.testing.assert_array_equal(orc["accepted_len"], [0, 1, 1])
     np.testing.assert_array_equal(st, orc["utt_status"] & 0xff)
     # tau <= 0 rejects nothing, tau >= 1 everything
-    out0 = run_verify(x.to(cuda_device), off, ids, V, 0.0, kernel=kernel)
+    out0 = run_verify(x.to(cuda_device), off, ids, V, 0.0, **kernel)
     assert list(out0["accepted_len"].cpu().numpy()) == [3, 3, 4]
-    out1 = run_verify(x.to(cuda_device), off, ids, V, 1.0, kernel=kernel)
+    out1 = run_verify(x.to(cuda_device), off, ids, V, 1.0, **kernel)
     assert list(out1["accepted_len"].cpu().numpy()) == [0, 0, 0]
+    # a draft token so dominant that fp32 rounds its log-likelihood to 0 or just above: tau = 1
+    # still rejects it (p <= 1)
+    x40 = x.clone()
+    for i in range(10):
+        x40[i, ids[i]] += 40.0
+    out40 = run_verify(x40.to(cuda_device), off, ids, V, 1.0, **kernel)
+    assert list(out40["accepted_len"].cpu().numpy()) == [0, 0, 0]
+    assert float(out40["token_logp"].abs().max()) < 1e-6
 
 
 @pytest.mark.parametrize("kernel", KERNELS.values(), ids=KERNELS.keys())
@@ -156,10 +173,10 @@ def test_exact_threshold_is_a_reject(cuda_device, kernel):
     x = torch.zeros((3, 2), dtype=torch.float32)
     ids = torch.tensor([0, 1, 0], dtype=torch.int32)
     off = torch.tensor([0, 3], dtype=torch.int64)
-    out = run_verify(x.to(cuda_device), off, ids, 2, 0.5, kernel=kernel)
+    out = run_verify(x.to(cuda_device), off, ids, 2, 0.5, **kernel)
     assert int(out["accepted_len"].cpu()[0]) == 0 and int(out["all_accepted"].cpu()[0]) == 0
     below = float(np.nextafter(np.float32(0.5), np.float32(0)))
-    out = run_verify(x.to(cuda_device), off, ids, 2, below, kernel=kernel)
+    out = run_verify(x.to(cuda_device), off, ids, 2, below, **kernel)
     assert int(out["accepted_len"].cpu()[0]) == 3 and int(out["all_accepted"].cpu()[0]) == 1
 
 
@@ -173,6 +190,27 @@ def test_empty_batch_and_malformed_offsets(cuda_device):
     out = run_verify(x.to(dev), off, ids, 9, 0.05)
     st = H.status_u32(out["utt_status"])
     assert st[1] == ssd.UTT_BAD_OFFSETS and int(out["all_accepted"].cpu()[1]) == 0
+
+
+@pytest.mark.parametrize("fill", [0x00, 0xff, 0x5a])
+def test_workspace_left_dirty_by_anything(cuda_device, fill):
+    """The words the streaming kernel keeps per utterance carry a per-call tag: whatever the
+    workspace held before, and on a second call that finds the first call's words, the outputs
+    are the oracle's."""
+    dev = cuda_device
+    w = synth.scaled(synth.CONFIGS[1], B=5, variant="literal", seed=71)
+    K = [19, 0, 31, 7, 12]
+    vb = synth.make_verify_batch(w, K, "cpu")
+    x, off, ids = vb.logits.to(dev), vb.tok_off.to(dev), vb.draft_ids.to(dev)
+    orc = ref.verify(H.storage_numpy(vb.logits), w.V_llm, vb.tok_off.numpy(), vb.draft_ids.numpy(),
+                     float(np.float32(w.tau_slm)))
+    out = ssd.alloc_verify_outputs(x.shape[0], 5, dev,
+                                   ssd.ssd_verify_workspace_bytes(5, x.shape[0], w.V_llm, ssd.BF16))
+    out["workspace"].fill_(fill)
+    for _ in range(2):
+        ssd.ssd_verify(x, off, ids, w.tau_slm, out=out)
+        torch.cuda.synchronize()
+        H.compare_stage2(out, orc, vb.tok_off.numpy(), w.tau_slm, require_all_margins=False)
 
 
 def test_runs_are_bit_identical(cuda_device):

@@ -113,3 +113,23 @@ def test_one_shard_reproduces_ssd_verify_bit_for_bit(cuda_device):
     for k in ("accepted_len", "all_accepted", "utt_status"):
         assert torch.equal(out[k], full[k]), k
     assert torch.allclose(out["token_logp"], full["token_logp"], rtol=0, atol=2e-6)
+
+
+def test_internal_error_mark_in_a_rank_statistics(cuda_device):
+    """The value a rank leaves in place of a row maximum when one of its kernel's bounded waits
+    ran out makes the combination report SSD_UTT_INTERNAL for that utterance."""
+    dev = cuda_device
+    M, R = 6, 2
+    st = torch.zeros((R, M, 3), dtype=torch.float32)
+    st[:, :, 0] = 1.0
+    st[:, :, 1] = 2.0
+    st[0, :, 2] = 1.0
+    st[1, :, 2] = -float("inf")
+    st[1, 4, 0] = torch.tensor([0x7fc0dead], dtype=torch.int32).view(torch.float32)[0]
+    off = torch.tensor([0, 3, 6], dtype=torch.int64, device=dev)
+    ids = torch.zeros(M, dtype=torch.int32, device=dev)
+    out = ssd.ssd_verify_combine(st.to(dev), 100, off, ids, 0.1)
+    torch.cuda.synchronize()
+    status = out["utt_status"].cpu().numpy().view(np.uint32)
+    assert status[0] == 0 and status[1] & ssd.UTT_INTERNAL
+    assert int(out["all_accepted"].cpu()[1]) == 0
