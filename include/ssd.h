@@ -79,9 +79,10 @@ typedef struct ssd_launch_opts {
                              0 auto; 1..3 that many of the 4 pairs (ctc_draft: at most 2);
                              -1 none */
     int32_t finish;       /* ssd_verify: where a row's log-likelihood and the utterance decisions
-                             are finished: 0 auto; 1 in a closing kernel of their own; 2 inside
-                             the streaming kernel (refused with SSD_ERR_ARG where that is not
-                             possible: column spans, the plain-load kernel, B > 2047) */
+                             are finished: 0 auto (the closing kernel); 1 in a closing kernel of
+                             their own; 2 inside the streaming kernel, one launch instead of two
+                             (refused with SSD_ERR_ARG where that is not possible: column spans,
+                             the plain-load kernel, B > 2047) */
 } ssd_launch_opts;
 
 /* Human-readable name of a return code (static storage). */

@@ -426,12 +426,6 @@ __global__ void __launch_bounds__(544, 1) verify_rows_fin(const FinParams q) {
                 const int64_t row = __shfl_sync(0xffffffffu, cur.row, src);
                 const int rslot = rowseq % NR;
                 ++rowseq;
-                if (lane == src) {
-                    FinRow rm;
-                    rm.row = cur.row; rm.b = cur.b; rm.pos = cur.pos;
-                    rm.id_ok = (cur.id >= 0 && cur.id < p.V) ? 1 : 0; rm.x = cur.x;
-                    rows[rslot] = rm;
-                }
                 const ranges::RowGeom geom = ranges::row_geom(
                     reinterpret_cast<uintptr_t>(p.logits), row, p.ld * ES, row_bytes);
                 const uintptr_t g0 = geom.g0, g1 = geom.g1, f0 = geom.f0;
@@ -492,6 +486,15 @@ __global__ void __launch_bounds__(544, 1) verify_rows_fin(const FinParams q) {
                     finalize(done_slot1);     // after the stage's next copy is under way
                     if (++s == S) { s = 0; ph ^= 1u; }
                 }
+                // what the row's finish needs; written after its copies are under way, since the
+                // draft id and logit of a kernel's first rows may still be on their way
+                if (lane == src) {
+                    FinRow rm;
+                    rm.row = cur.row; rm.b = cur.b; rm.pos = cur.pos;
+                    rm.id_ok = (cur.id >= 0 && cur.id < p.V) ? 1 : 0; rm.x = cur.x;
+                    rows[rslot] = rm;
+                }
+                __syncwarp();
             }
         }
         if (!failed) {
@@ -875,12 +878,15 @@ int plan_verify(int B, int64_t M, int V, ssd_dtype dtype, const ssd_launch_opts 
     // header | two words per utterance | partials
     pl.workspace_bytes = 256 + (((size_t)(B > 0 ? B : 0) * 16 + 255) & ~(size_t)255) +
                          (size_t)M * pl.partials * sizeof(float2);
-    // rows are finished inside the streaming kernel where that kernel sees whole rows and can
-    // keep the utterance offsets in shared memory
+    // Rows can be finished inside the streaming kernel where that kernel sees whole rows and can
+    // keep the utterance offsets in shared memory.  It is not the default: in a chain of calls
+    // the closing kernel's few microseconds are when the next streaming kernel's CTAs (which
+    // need the SM's whole shared memory) get resident and past their set-up, and without it that
+    // ramp-up is exposed instead (measured: 108 against 104 us per step on 32 utterances).
     const int finish = o ? o->finish : 0;
     if (finish < 0 || finish > 2) return SSD_ERR_ARG;
     pl.finish_inside = 0;
-    if (finish != 1 && pl.kernel == 2 && split == 1 && B > 0 && B + 1 <= kOffCacheMax && M > 0) {
+    if (finish == 2 && pl.kernel == 2 && split == 1 && B > 0 && B + 1 <= kOffCacheMax && M > 0) {
         const int NR = 2 * pl.stages;
         size_t hdr = 2 * (size_t)pl.stages * 8 + pl.stages * sizeof(StageDesc) + NR * sizeof(FinRow) +
                      (size_t)NR * pl.warps * 8 + pl.stages * 4 + 8 + (size_t)(B + 1) * 8;

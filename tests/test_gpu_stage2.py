@@ -109,8 +109,9 @@ def test_column_spans(cuda_device, dtype, split):
                                                             (8, 12, 16384, 7), (1, 16, 1024, 1)])
 def test_pipeline_shapes(cuda_device, warps, stages, stage_bytes, ctas):
     w = synth.scaled(synth.CONFIGS[1], B=4, V_llm=32000, seed=17)
-    check_verify(w, [11, 3, 8, 5], cuda_device, 2, warps=warps, stages=stages,
-                 stage_bytes=stage_bytes, ctas=ctas)
+    for extra in (dict(finish=1), dict(finish=2, split=1)):
+        check_verify(w, [11, 3, 8, 5], cuda_device, 2, warps=warps, stages=stages,
+                     stage_bytes=stage_bytes, ctas=ctas, **extra)
 
 
 @pytest.mark.parametrize("kernel", KERNELS.values(), ids=KERNELS.keys())
@@ -205,10 +206,11 @@ def test_workspace_left_dirty_by_anything(cuda_device, fill):
     orc = ref.verify(H.storage_numpy(vb.logits), w.V_llm, vb.tok_off.numpy(), vb.draft_ids.numpy(),
                      float(np.float32(w.tau_slm)))
     out = ssd.alloc_verify_outputs(x.shape[0], 5, dev,
-                                   ssd.ssd_verify_workspace_bytes(5, x.shape[0], w.V_llm, ssd.BF16))
+                                   ssd.ssd_verify_workspace_bytes(5, x.shape[0], w.V_llm, ssd.BF16,
+                                                                  H.opts(finish=2, split=1)))
     out["workspace"].fill_(fill)
     for _ in range(2):
-        ssd.ssd_verify(x, off, ids, w.tau_slm, out=out)
+        ssd.ssd_verify(x, off, ids, w.tau_slm, out=out, opts=H.opts(finish=2, split=1))
         torch.cuda.synchronize()
         H.compare_stage2(out, orc, vb.tok_off.numpy(), w.tau_slm, require_all_margins=False)
 
