@@ -320,6 +320,7 @@ __device__ __forceinline__ void reduce_tile(const CtcParams &p, uint32_t stage_a
     constexpr uint32_t STEP = (uint32_t)G * 16;
     const int sub = lane % G, grp = lane / G;
     const uint32_t pitch = (uint32_t)(p.ld * ES), row_bytes = (uint32_t)p.V * ES;
+    constexpr int kDepth = 8;       // interior chunks in flight per lane
     const int ITER = p.iters, KT = p.tail_from;
     for (int g0 = 0; g0 < nrows; g0 += RPW) {
         const int i = g0 + grp;
@@ -362,6 +363,21 @@ __device__ __forceinline__ void reduce_tile(const CtcParams &p, uint32_t stage_a
         }
         a += STEP; c += G;
         int k = 1;
+        {
+            // kDepth chunks in flight: with at most 16 warps per SM (128 registers each) the
+            // arithmetic hides its own latencies only if a warp has many independent chunks
+            // to work on (four in flight at 24 warps and 80 registers ran 8 % slower)
+#pragma unroll 1
+            for (; k + kDepth <= KT; k += kDepth) {
+                uint4 w[kDepth];
+#pragma unroll
+                for (int j = 0; j < kDepth; ++j) w[j] = lds128(a + j * STEP);
+#pragma unroll
+                for (int j = 0; j < kDepth; ++j)
+                    FusedChunk<T, kF>::run(w[j], c + j * G, nrh, floor2, vmax, vc, Sa, Sb, Aa, Ab);
+                a += kDepth * STEP; c += kDepth * G;
+            }
+        }
 #pragma unroll 1
         for (; k + 4 <= KT; k += 4) {           // interior chunks, four in flight
             const uint4 w0 = lds128(a), w1 = lds128(a + STEP), w2 = lds128(a + 2 * STEP),
@@ -468,7 +484,7 @@ __device__ __forceinline__ MaxAt warp_max_at(MaxAt x) {
 // same number of tiles and of warps and run out together.  The claim for the tile after the
 // current one is in flight while the current one is worked on.
 template <typename T, int G, int kF>
-__global__ void __launch_bounds__(768, 1) ctc_rows_tma(const CtcParams p) {
+__global__ void __launch_bounds__(512, 1) ctc_rows_tma(const CtcParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     constexpr int ES = Elem<T>::kBytes, EPC = Elem<T>::kPerChunk;
     pdl_launch_dependents();
@@ -839,7 +855,7 @@ int plan_ctc(ssd_dtype dtype, int V, int64_t ld, int64_t N, int B, const ssd_lau
     if (tail_from < 1) tail_from = 1;
     (void)B;
     const int epc = 16 / es;
-    const int64_t fixed = 24 * 8 + 16 + (int64_t)epc * (epc + 1) * 16 + 128;
+    const int64_t fixed = 16 * 8 + 16 + (int64_t)epc * (epc + 1) * 16 + 128;
     const int64_t stage_budget = 216 * 1024 - fixed;
     int warps = 0, R = 0;
     int64_t stage_stride = 0;
@@ -853,7 +869,7 @@ int plan_ctc(ssd_dtype dtype, int V, int64_t ld, int64_t N, int B, const ssd_lau
             // the row reaches that far or not (what lies past it is masked, not used)
             stage_stride = ((R - 1) * row_pitch + 16 + (int64_t)iters * G * 16 + 127) & ~127ll;
             int64_t w = stage_budget / stage_stride;
-            if (w > 24) w = 24;
+            if (w > 16) w = 16;      // 512 threads: 128 registers each, for eight chunks in flight
             if (w >= 5 && w % 2 && w % 3) --w;      // so that 2 or more tile counters divide it
             if (o && o->warps > 0 && o->warps < w) w = o->warps;
             if (w >= 1) warps = (int)w;
