@@ -39,7 +39,7 @@ struct CtcParams {
     int32_t *frame_argmax;
     float *frame_lse;
     float *frame_logprob;
-    // tiles are handed out from kTileCounters counters in the caller's workspace, 256 bytes
+    // tiles are handed out from up to four counters in the caller's workspace, 256 bytes
     // apart (NULL: tile j to warp j mod the number of warps).  A word is {epoch : 32 | count :
     // 32}, so a call needs no clearing of what the last one left there.
     unsigned long long *tile_counter;
@@ -47,7 +47,6 @@ struct CtcParams {
     int counters;          // C
     int claim;             // tiles per claim
 };
-constexpr int kTileCounters = 4;      // at most; a launch uses the largest divisor of its warps per CTA
 
 // Replaces the elements of a 16-byte chunk outside [e_lo, e_hi) (they belong to a neighbouring
 // row, to the padding between rows, or were never written) by -inf.
