@@ -85,12 +85,12 @@ __device__ __forceinline__ void load_u8_if(int &dst, const uint8_t *ptr, bool pr
     asm volatile("{ .reg .pred q; setp.ne.s32 q, %2, 0; @q ld.global.u8 %0, [%1]; }"
                  : "+r"(dst) : "l"(ptr), "r"((int)pred) : "memory");
 }
-// Whether the phase has completed, without waiting (try_wait may keep the thread for a time of
-// the hardware's choosing: microseconds when nothing completes the phase).
-__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+// try_wait that gives the thread back after about `ns` nanoseconds at the latest (the plain form
+// may keep it for a time of the hardware's choosing: microseconds when nothing completes the phase).
+__device__ __forceinline__ bool mbar_try_wait_for(uint32_t bar, uint32_t parity, uint32_t ns) {
     uint32_t ok;
-    asm volatile("{ .reg .pred q; mbarrier.test_wait.parity.shared::cta.b64 q, [%1], %2; selp.u32 %0, 1, 0, q; }"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    asm volatile("{ .reg .pred q; mbarrier.try_wait.parity.shared::cta.b64 q, [%1], %2, %3; selp.u32 %0, 1, 0, q; }"
+                 : "=r"(ok) : "r"(bar), "r"(parity), "r"(ns) : "memory");
     return ok != 0;
 }
 __device__ __forceinline__ void atom_add_u64_if(unsigned long long &dst, unsigned long long *ptr,
@@ -432,18 +432,19 @@ __global__ void __launch_bounds__(576, 1) verify_rows_ee(const EeParams p) {
         for (int seq = 0;; ++seq) {
             const int slot = seq % NR;
             const uint32_t bar = rowdone0 + slot * 8, par = (uint32_t)((seq / NR) & 1);
-            // Polls, rather than waits, for the row: after the last row nothing completes the
-            // barrier, and a waiting form would sit out its time before the end is noticed
-            // (measured: the kernel ended 4 us after its last row).
+            // Sleeps on the row's barrier half a microsecond at a time, looking for the end in
+            // between.  (After the last row nothing completes the barrier: the plain wait sat out
+            // its time there and the kernel ended 4 us after its last row; and a loop that only
+            // tests the barrier keeps a warp spinning on every SM, which under the power cap cost
+            // 3 % of the clock.)
             bool got = false;
             const long long t0 = clock64();
             for (;;) {
-                got = __all_sync(0xffffffffu, mbar_test_wait(bar, par));
+                got = __all_sync(0xffffffffu, mbar_try_wait_for(bar, par, 500u));
                 if (got) break;
                 const int e = __shfl_sync(0xffffffffu, (int)*end_seq, 0);
                 if (e == kEeAborted || (e >= 0 && seq >= e)) break;
                 if (__any_sync(0xffffffffu, clock64() - t0 > kWaitLimitCycles)) { failed = true; break; }
-                __nanosleep(64);
             }
             if (!got) break;
             const float2 v = lane < CW ? spart[slot * CW + lane] : make_float2(kNegInit, 0.f);
