@@ -290,6 +290,18 @@ def test_early_exit_shapes_skip_and_ragged(cuda_device, dtype, V):
     check_early_exit(w, K, cuda_device, skip=None, warps=4, stages=3, stage_bytes=4096, ctas=7)
 
 
+def test_early_exit_thousands_of_short_utterances(cuda_device):
+    """More utterances than the kernel keeps offsets for in shared memory, rows so short that the
+    warp that finishes rows is what limits the rate (its hand-back of row slots holds the
+    producer), drafts of 0 to 4 tokens."""
+    B = 2500
+    w = synth.scaled(synth.CONFIGS[3], B=B, V_llm=96, seed=77)
+    K = [(7 * i + i // 5) % 5 for i in range(B)]
+    vb, out, orc, rr = check_early_exit(w, K, cuda_device, ctas=24)
+    assert (rr >= 0).all()                                   # the position-major kernel ran
+    assert int(rr.sum()) <= sum(K)
+
+
 def test_early_exit_falls_back_on_small_batches(cuda_device):
     w = synth.scaled(synth.CONFIGS[1], B=3, V_llm=32000, seed=9)
     vb, out, orc, rr = check_early_exit(w, [12, 30, 7], cuda_device)
