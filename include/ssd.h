@@ -24,6 +24,13 @@
  *     (nothing is written in that case).  Problems only visible in the data are reported
  *     per utterance in `utt_status` (bit set, no trap, nothing out of bounds is touched).
  *   - Ties of the argmax go to the lowest index.  Entropy is in nats.
+ *   - CUDA graphs: every call only enqueues kernels on `stream` and may be captured into a
+ *     graph and replayed with new contents in the same buffers.  Make one call of each kind,
+ *     with the same sizes, before capturing (the first use of a kernel sets a function
+ *     attribute and looks up device properties).  What a replay cannot renew is the call
+ *     number that marks a workspace's error word: after a replay that reported
+ *     SSD_UTT_INTERNAL, later replays of the same graph report it too; capture again.
+ *     ssd_verify with opts->finish == 2 is refused (SSD_ERR_ARG) while its stream is capturing.
  */
 #ifndef SSD_H_
 #define SSD_H_
@@ -82,7 +89,7 @@ typedef struct ssd_launch_opts {
                              are finished: 0 auto (the closing kernel); 1 in a closing kernel of
                              their own; 2 inside the streaming kernel, one launch instead of two
                              (refused with SSD_ERR_ARG where that is not possible: column spans,
-                             the plain-load kernel, B > 2047) */
+                             the plain-load kernel, B > 2047, a stream that is capturing) */
 } ssd_launch_opts;
 
 /* Human-readable name of a return code (static storage). */

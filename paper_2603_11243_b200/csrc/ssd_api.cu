@@ -133,7 +133,7 @@ int32_t ssd_ctc_draft(const void *logits, ssd_dtype dtype, int32_t V, int64_t ld
     if (rc != SSD_OK) return rc;
     return launch_collapse(frame_argmax, frame_entropy, frame_off, B, N, blank_id, max_draft_len,
                            draft_tokens, draft_frames, draft_len, draft_full_len,
-                           utt_max_entropy, utt_status, L.stream);
+                           utt_max_entropy, utt_status, workspace, L.stream);
 }
 
 int32_t ssd_entropy_gate(const float *frame_entropy, const int64_t *frame_off,

@@ -382,7 +382,7 @@ int launch_collapse(const int32_t *frame_argmax, const float *frame_entropy,
                     const int64_t *frame_off, int B, int64_t N, int blank_id, int max_draft_len,
                     int32_t *draft_tokens, int32_t *draft_frames, int32_t *draft_len,
                     int32_t *draft_full_len, float *utt_max_entropy, uint32_t *utt_status,
-                    cudaStream_t stream);
+                    void *workspace, cudaStream_t stream);
 int launch_gate(const float *frame_entropy, const int64_t *frame_off, int B, int64_t N,
                 float tau, uint8_t *gate_accept, float *max_entropy, int32_t *argmax_frame,
                 cudaStream_t stream);

@@ -43,6 +43,7 @@ struct CtcParams {
     // apart (NULL: tile j to warp j mod the number of warps).  A word is {epoch : 32 | count :
     // 32}, so a call needs no clearing of what the last one left there.
     unsigned long long *tile_counter;
+    const unsigned long long *launch_gen;   // launches this workspace has seen (see launch_ctc_rows)
     uint32_t epoch;
     int counters;          // C
     int claim;             // tiles per claim
@@ -543,6 +544,7 @@ __global__ void __launch_bounds__(512, 1) ctc_rows_tma(const CtcParams p) {
     };
 
     const bool dynamic = p.tile_counter != nullptr && p.num_tiles > GW;
+    uint32_t epoch = p.epoch;
     const int C = p.counters;
     unsigned long long *counter = p.tile_counter + (warp % C) * 32;
     const int64_t first = GW + warp % C;                 // tile of this counter's slot 0
@@ -554,11 +556,18 @@ __global__ void __launch_bounds__(512, 1) ctc_rows_tma(const CtcParams p) {
     uint32_t pend_k = 0;
     auto claim_begin = [&]() {
         pend_k = p.claim;
-        if (lane == 0) pend = tagged_begin(counter, p.epoch, pend_k);
+        if (lane == 0) pend = tagged_begin(counter, epoch, pend_k);
     };
     pdl_wait();
     issue(t);
-    if (dynamic) claim_begin();
+    if (dynamic) {
+        // The tag of this launch's counter words: the host's call number plus the number of
+        // launches the workspace has seen, so that a launch that is replayed with the same
+        // parameters (a captured graph) does not take the counts of the replay before it for
+        // its own.
+        epoch += (uint32_t)__ldcg(p.launch_gen);
+        claim_begin();
+    }
     while (t < p.num_tiles) {
         if (!mbar_wait_bounded(bar, parity)) { failed = true; break; }
         parity ^= 1u;
@@ -571,7 +580,7 @@ __global__ void __launch_bounds__(512, 1) ctc_rows_tma(const CtcParams p) {
         if (dynamic && nt >= t_end) {
             // the claimed tiles are used up: take the claim in flight, start the next one
             uint32_t cnt = 0;
-            if (lane == 0) cnt = tagged_finish(counter, p.epoch, pend_k, pend, ok);
+            if (lane == 0) cnt = tagged_finish(counter, epoch, pend_k, pend, ok);
             cnt = __shfl_sync(0xffffffffu, cnt, 0);
             if (!__shfl_sync(0xffffffffu, (int)ok, 0)) { failed = true; break; }
             step = C;
@@ -598,7 +607,7 @@ __global__ void __launch_bounds__(512, 1) ctc_rows_tma(const CtcParams p) {
         if (dynamic) {
             // the claim in flight: its tiles are this warp's as well
             uint32_t cnt = 0xffffffffu;
-            if (lane == 0 && (uint32_t)(pend >> 32) == p.epoch) cnt = (uint32_t)pend;
+            if (lane == 0 && (uint32_t)(pend >> 32) == epoch) cnt = (uint32_t)pend;
             cnt = __shfl_sync(0xffffffffu, cnt, 0);
             if (cnt != 0xffffffffu) {
                 t = first + (int64_t)cnt * C;
@@ -686,13 +695,16 @@ __global__ void __launch_bounds__(kUttThreads) collapse_kernel(
     const int64_t *__restrict__ frame_off, int B, int64_t N, int blank_id, int cap,
     int32_t *__restrict__ draft_tokens, int32_t *__restrict__ draft_frames,
     int32_t *__restrict__ draft_len, int32_t *__restrict__ draft_full_len,
-    float *__restrict__ utt_max_entropy, uint32_t *__restrict__ utt_status) {
+    float *__restrict__ utt_max_entropy, uint32_t *__restrict__ utt_status,
+    unsigned long long *launch_gen) {
     __shared__ int warp_tot[2][32];
     __shared__ MaxAt scratch[32];
     __shared__ unsigned flags_sh[32];
     pdl_enter();
     const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nw = blockDim.x >> 5;
+    // the frame statistics kernel before this one is through, the next one has not begun
+    if (launch_gen && b == 0 && tid == 0) *launch_gen = *launch_gen + 1;
     const int64_t t0 = frame_off[b], t1 = frame_off[b + 1];
     if (t0 < 0 || t1 < t0 || t1 > N) {
         if (tid == 0) {
@@ -927,7 +939,9 @@ int launch_ctc_rows(const void *logits, ssd_dtype dtype, int V, int64_t ld, int6
         p.stage_stride = plan.stage_stride;
         p.iters = plan.iters; p.tail_from = plan.tail_from;
         p.num_tiles = (N + R - 1) / R;
+        // workspace: four counter words 256 bytes apart, then the launch count at byte 1024
         p.tile_counter = static_cast<unsigned long long *>(workspace);
+        p.launch_gen = workspace ? static_cast<unsigned long long *>(workspace) + 128 : nullptr;
         p.epoch = (uint32_t)next_epoch();
         p.counters = plan.warps % 4 == 0 ? 4 : plan.warps % 3 == 0 ? 3 : plan.warps % 2 == 0 ? 2 : 1;
         // small tiles are finished faster than a counter hands them out one by one
@@ -969,11 +983,13 @@ int launch_collapse(const int32_t *frame_argmax, const float *frame_entropy,
                     const int64_t *frame_off, int B, int64_t N, int blank_id, int max_draft_len,
                     int32_t *draft_tokens, int32_t *draft_frames, int32_t *draft_len,
                     int32_t *draft_full_len, float *utt_max_entropy, uint32_t *utt_status,
-                    cudaStream_t stream) {
+                    void *workspace, cudaStream_t stream) {
     if (B == 0) return SSD_OK;
+    unsigned long long *launch_gen =
+        workspace ? static_cast<unsigned long long *>(workspace) + 128 : nullptr;
     cudaError_t e = launch_pdl(collapse_kernel, (unsigned)B, (unsigned)kUttThreads, 0, stream,
         frame_argmax, frame_entropy, frame_off, B, N, blank_id, max_draft_len, draft_tokens,
-        draft_frames, draft_len, draft_full_len, utt_max_entropy, utt_status);
+        draft_frames, draft_len, draft_full_len, utt_max_entropy, utt_status, launch_gen);
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
     return SSD_OK;

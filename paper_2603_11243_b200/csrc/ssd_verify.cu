@@ -978,6 +978,12 @@ int launch_verify(const void *logits, ssd_dtype dtype, int V, int64_t ld, int64_
     const Threshold th = threshold_of(tau_slm);
     cudaError_t e;
     if (plan.finish_inside) {
+        // The per-utterance words of this variant are told apart from leftovers by the host's
+        // call number, which a captured launch would repeat at every replay: not while capturing.
+        cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+        e = cudaStreamIsCapturing(L.stream, &capturing);
+        if (e != cudaSuccess) { record_cuda_error(e); return SSD_ERR_CUDA; }
+        if (capturing != cudaStreamCaptureStatusNone) return SSD_ERR_ARG;
         FinParams q{};
         VerifyParams &p = q.v;
         p.logits = static_cast<const char *>(logits);
