@@ -95,6 +95,37 @@ def global_properties(w, cb, vb, s1, gate, s2, K):
     assert (lp[rows] <= 1e-5).all() and np.isfinite(lp[rows]).all()
 
 
+def early_exit_agrees(w, vb, gate, s2, dev):
+    """ssd_verify_early_exit on the same rows: the same decisions, log-likelihoods up to each
+    first reject that agree with ssd_verify's, and no more rows read than there are."""
+    off, ids = vb.tok_off.to(dev), vb.draft_ids.to(dev)
+    M, B = vb.logits.shape[0], w.B
+    code = ssd.BF16 if vb.logits.dtype == torch.bfloat16 else ssd.F32
+    out = ssd.alloc_early_exit_outputs(M, B, w.V_llm, code, dev)
+    out["token_logp"].fill_(float("nan"))
+    ssd.ssd_verify_early_exit(vb.logits, off, ids, w.tau_slm, skip=gate["gate_accept"], out=out)
+    torch.cuda.synchronize()
+    for k in ("accepted_len", "all_accepted", "utt_status"):
+        assert torch.equal(out[k], s2[k]), k
+    rr = out["rows_read"].cpu().numpy()
+    K = np.diff(vb.tok_off.numpy())
+    ga = gate["gate_accept"].cpu().numpy().astype(bool)
+    al = s2["accepted_len"].cpu().numpy()
+    assert (rr >= 0).all(), "the position-major kernel did not run"
+    assert (rr[ga] == 0).all() and (rr <= K).all()
+    assert (rr[~ga] >= np.minimum(K, al + 1)[~ga]).all()
+    lp_e, lp_f = out["token_logp"].cpu().numpy(), s2["token_logp"].cpu().numpy()
+    read = ~np.isnan(lp_e)
+    assert read.sum() == rr.sum()
+    assert np.abs(lp_e[read] - lp_f[read]).max(initial=0.0) <= 1e-5
+    # every position up to the first reject was read
+    toff = vb.tok_off.numpy()
+    for b in np.flatnonzero(~ga):
+        need = min(int(K[b]), int(al[b]) + 1)
+        assert read[toff[b]:toff[b] + need].all()
+    return float(rr.sum()) / max(1, int(K[~ga].sum()))
+
+
 def pick(T, ga, n):
     order = np.argsort(T)
     sample = {int(order[0]), int(order[-1]), int(order[len(order) // 2])}
@@ -112,6 +143,7 @@ def test_configuration1_every_output(cuda_device):
     cb, vb, s1, gate, s2, K = run_path(w, cuda_device)
     global_properties(w, cb, vb, s1, gate, s2, K)
     check_sample(w, cb, vb, s1, gate, s2, range(w.B))
+    assert early_exit_agrees(w, vb, gate, s2, cuda_device) < 0.9
 
 
 @pytest.mark.parametrize("cfg,n_sample", [(2, 6), (3, 6)])
@@ -123,6 +155,7 @@ def test_configurations_2_and_3_sampled(cuda_device, cfg, n_sample):
     T = np.diff(cb.frame_off.numpy())
     sample = pick(T, gate["gate_accept"].cpu().numpy(), n_sample)
     check_sample(w, cb, vb, s1, gate, s2, sample)
+    assert early_exit_agrees(w, vb, gate, s2, cuda_device) < 0.8
     del cb, vb, s1, gate, s2
     torch.cuda.empty_cache()
 
