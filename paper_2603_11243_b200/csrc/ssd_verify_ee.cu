@@ -74,9 +74,10 @@ constexpr int kEeRunning = -1, kEeAborted = -2;     // end_seq before the produc
 constexpr uint32_t kFlagFirst = 4u;                 // stage flag: first stage of a row
 
 // Loads and the claim's atomic as the producer issues them: under a predicate, straight into a
-// register that already holds the value for "not loaded".  Written as `if (c) v = load` they
-// came out with the result copied at the join, which made the warp wait for the memory there
-// and then (measured: 1,100 cycles for a claim whose value is not needed for two rows' time).
+// register that already holds the value for "not loaded".  Written as `if (c) v = load` the warp
+// was found waiting for the memory right there (by cycle counter: 1,100 cycles for a claim whose
+// value is not needed for two rows' time), as if the result were copied where the branches
+// join; issued this way it waits where the value is used.
 __device__ __forceinline__ void load_volatile_s32_if(int &dst, const int32_t *ptr, bool pred) {
     asm volatile("{ .reg .pred q; setp.ne.s32 q, %2, 0; @q ld.volatile.global.s32 %0, [%1]; }"
                  : "+r"(dst) : "l"(ptr), "r"((int)pred) : "memory");
