@@ -215,8 +215,9 @@ int32_t ssd_verify(const void *logits, ssd_dtype dtype, int32_t V, int64_t ld,
  * Section 2.3 of the paper needs only j, the FIRST position whose likelihood is <= tau_SLM:
  * the rows after it cannot change the decision.  Rows are visited position by position across
  * all utterances; a row is skipped when a smaller rejected position of its utterance has
- * already been found.  accepted_len, all_accepted and utt_status are exactly those of
- * ssd_verify (status bits only reflect the rows that were read).  token_logp / row_lse are
+ * already been found.  accepted_len and all_accepted are exactly those of ssd_verify;
+ * utt_status has those of ssd_verify's bits that the rows read give rise to (a NaN or a bad
+ * draft id in a row after the first reject goes unseen).  token_logp / row_lse are
  * written for every row that was read -- always including positions 0 .. accepted_len[b] --
  * and left untouched for the others; which later rows still get read depends on timing.
  *   rows_read[b] (nullable, [B] i32): rows of utterance b that were read; -1 for every

@@ -238,3 +238,66 @@ def test_huge_dynamic_range_takes_the_redo_paths(cuda_device, dtype, scale):
     np.testing.assert_array_equal(gr["next_token"].cpu().numpy(), og["next_token"])
     _close_scaled(gr["next_logp"].cpu().numpy(), og["next_logp"], "next_logp")
     _close_scaled(gr["row_lse"].cpu().numpy(), og["row_lse"], "greedy row_lse")
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_early_exit_against_verify_random_options(cuda_device, seed):
+    """Random shapes, thresholds, skip flags and launch options (grid, warps, ring): the same
+    decisions as ssd_verify, its log-likelihoods up to each first reject, and no status bit that
+    ssd_verify does not report (bits of rows after a first reject may be missing: not read)."""
+    rng = np.random.default_rng(7000 + seed)
+    V = int(rng.choice([33, 257, 1000, 4099, 8192, 16384]))
+    dtype = torch.bfloat16 if rng.random() < 0.6 else torch.float32
+    B = int(rng.choice([1, 2, 7, 32, 33, 257, 2049]))
+    lens = rng.integers(0, int(rng.choice([3, 10, 60, 200])) + 1, size=B)
+    ctas = int(rng.choice([0, 8, 37]))
+    while lens.sum() < 4 * (ctas if ctas else 148) + 5:
+        lens = lens + 1 + rng.integers(0, 3, size=B)
+    off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    M = int(off[-1])
+    dev = cuda_device
+    g = torch.Generator(device=dev)
+    g.manual_seed(seed)
+    pad = int(rng.integers(0, 9))
+    col0 = int(rng.integers(0, pad + 1))
+    wide = (torch.randn((M, V + pad), generator=g, device=dev) * 2).to(dtype)
+    ids = torch.randint(0, V, (M,), generator=g, device=dev, dtype=torch.int32)
+    keep = torch.rand((M,), generator=g, device=dev) < float(rng.choice([0.9, 0.97, 0.995, 1.0]))
+    rows = torch.arange(M, device=dev)[keep]
+    wide[rows, col0 + ids[rows].long()] = 30.0
+    if rng.random() < 0.3:
+        ids[int(rng.integers(0, M))] = V + 3
+    view = wide[:, col0:col0 + V]
+    offd = torch.from_numpy(off).to(dev)
+    skip = (torch.rand((B,), generator=g, device=dev) < 0.3).to(torch.uint8) if rng.random() < 0.5 else None
+    kw = {}
+    if ctas:
+        kw["ctas"] = ctas
+    if rng.random() < 0.4:
+        kw["warps"] = int(rng.choice([1, 3, 4, 8, 12, 16]))
+    if rng.random() < 0.4:
+        kw["stage_bytes"], kw["stages"] = int(rng.choice([1024, 4096, 16384, 32768])), int(rng.choice([2, 3, 5, 9]))
+    o = H.opts(**kw) if kw else None
+    tau = float(rng.choice([0.1, 0.2, 0.0, 1.0, 0.5]))
+    try:
+        full = ssd.ssd_verify(view, offd, ids, tau, skip=skip, V=V, opts=o)
+    except ssd.SsdError as e:
+        assert e.code == ssd.ERR_ARG          # a ring that does not fit: refused on the host
+        return
+    ee = ssd.ssd_verify_early_exit(view, offd, ids, tau, skip=skip, V=V, opts=o)
+    torch.cuda.synchronize()
+    assert torch.equal(ee["accepted_len"], full["accepted_len"])
+    assert torch.equal(ee["all_accepted"], full["all_accepted"])
+    se, sf = H.status_u32(ee["utt_status"]), H.status_u32(full["utt_status"])
+    assert not (se & ~sf).any() and not (sf & 0x80000000).any()
+    rr = ee["rows_read"].cpu().numpy()
+    assert (rr >= 0).all()
+    assert (se[rr == lens] == sf[rr == lens]).all()
+    al = full["accepted_len"].cpu().numpy()
+    sk = skip.cpu().numpy().astype(bool) if skip is not None else np.zeros(B, bool)
+    a, c = ee["token_logp"].cpu().numpy(), full["token_logp"].cpu().numpy()
+    for b in np.flatnonzero(~sk):
+        s = slice(int(off[b]), int(off[b]) + min(int(lens[b]), int(al[b]) + 1))
+        fin = np.isfinite(c[s])
+        assert np.abs(a[s][fin] - c[s][fin]).max(initial=0.0) <= 2e-5
+        np.testing.assert_array_equal(a[s][~fin], c[s][~fin])
