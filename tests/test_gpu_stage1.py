@@ -235,6 +235,36 @@ def test_short_rows_far_from_zero(cuda_device, dtype, V, shift):
         H.compare_stage1(out, gate, orc, cb.frame_off.numpy(), 0.9, require_all_margins=False)
 
 
+@pytest.mark.parametrize("V,shift", [(5000, -150.0), (4097, 90.0), (20000, -150.0)])
+def test_one_logit_far_above_many_equal_ones(cuda_device, V, shift):
+    """bf16 rows far from zero, where a step of the format is 1: the many small logits take three
+    or four values, one logit stands 12 above them.  A lane's running sums then hold one term of
+    2^17 and get thousands of equal small ones added, whose rounding errors all point the same
+    way unless they are summed apart first.  With few lanes per row (long lanes) this was off
+    by 1.4e-4; half the tolerance is asked for here."""
+    g = torch.Generator().manual_seed(V)
+    T = [130, 0, 75, 1]
+    N = sum(T)
+    x = torch.randn((N, V), generator=g) * 0.3 + shift
+    win = torch.randint(0, V, (N,), generator=g)
+    x[torch.arange(N), win] += 12.0
+    x = x.to(torch.bfloat16)
+    off = torch.tensor([0] + list(np.cumsum(T)), dtype=torch.int64)
+    orc = H.oracle_stage1(H.storage_numpy(x), V, off.numpy(), 0, 50, 0.9)
+    ran = 0
+    for G in (0, 4, 8, 16, 32):
+        try:
+            out, gate = run_stage1(x.to(cuda_device), off, V, 0, 50, 0.9, 2, split=G)
+        except ssd.SsdError as e:
+            assert e.code == ssd.ERR_ARG and G != 0      # too many chunks per lane: refused
+            continue
+        ran += 1
+        H.compare_stage1(out, gate, orc, off.numpy(), 0.9, require_all_margins=False)
+        dH = np.abs(out["frame_entropy"].cpu().numpy().astype(np.float64) - orc["frame_entropy"])
+        assert dH.max() <= 0.5 * H.FLOAT_TOL, (G, dH.max())
+    assert ran >= 2
+
+
 @pytest.mark.parametrize("V,dtype", [(1025, "bf16"), (348, "bf16"), (4097, "bf16"), (129, "f32"),
                                      (1025, "f32"), (2049, "bf16"), (64, "bf16"), (7, "bf16")])
 def test_lanes_per_row_and_exponential_split(cuda_device, V, dtype):
