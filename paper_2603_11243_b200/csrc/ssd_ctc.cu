@@ -572,7 +572,7 @@ __global__ void __launch_bounds__(512, 1) ctc_rows_tma(const CtcParams p) {
         // launches the workspace has seen, so that a launch that is replayed with the same
         // parameters (a captured graph) does not take the counts of the replay before it for
         // its own.
-        epoch += (uint32_t)__ldcg(p.launch_gen);
+        epoch = scratch_tag(epoch + (uint32_t)__ldcg(p.launch_gen));
         claim_begin();
     }
     while (t < p.num_tiles) {

@@ -997,7 +997,7 @@ int launch_verify(const void *logits, ssd_dtype dtype, int V, int64_t ld, int64_
         q.accepted_len = accepted_len; q.all_accepted = all_accepted; q.utt_status = utt_status;
         q.utt_words = reinterpret_cast<unsigned long long *>(static_cast<char *>(workspace) + 256);
         q.done_ctas = err_word + 1;
-        q.epoch32 = (uint32_t)epoch;
+        q.epoch32 = scratch_tag((uint32_t)epoch);
         const int64_t ctas = M < plan.ctas ? M : plan.ctas;
         if (o && o->ev_begin) {
             e = cudaEventRecord(static_cast<cudaEvent_t>(o->ev_begin), L.stream);
