@@ -301,3 +301,119 @@ def test_early_exit_against_verify_random_options(cuda_device, seed):
         fin = np.isfinite(c[s])
         assert np.abs(a[s][fin] - c[s][fin]).max(initial=0.0) <= 2e-5
         np.testing.assert_array_equal(a[s][~fin], c[s][~fin])
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_frame_statistics_kernels_agree_under_random_options(cuda_device, seed):
+    """The bulk-copy kernel under random launch options (grid, warps, lanes per row, where the
+    exponentials run) against the plain-load kernel: rows of 1 to 5,000 symbols, ragged batches,
+    logits far from zero, views with padded rows."""
+    rng = np.random.default_rng(8000 + seed)
+    V = int(rng.choice([1, 7, 33, 129, 348, 1025, 4097, 5000]))
+    dtype = torch.bfloat16 if rng.random() < 0.6 else torch.float32
+    B = int(rng.choice([1, 3, 17, 64, 300, 2500]))
+    T = rng.integers(0, int(rng.choice([5, 40, 400])) + 1, size=B)
+    N = int(T.sum())
+    if N == 0 or N * V > 1e8:
+        T = np.minimum(T, 3) + (np.arange(B) == 0)
+        N = int(T.sum())
+    dev = cuda_device
+    off = torch.from_numpy(np.concatenate([[0], np.cumsum(T)]).astype(np.int64)).to(dev)
+    pad = int(rng.integers(0, 9))
+    col0 = int(rng.integers(0, pad + 1))
+    g = torch.Generator(device=dev)
+    g.manual_seed(seed)
+    shift, scale = float(rng.choice([0.0, 0.0, -150.0, 90.0])), float(rng.choice([0.3, 2.0, 8.0]))
+    wide = (torch.randn((N, V + pad), generator=g, device=dev) * scale + shift).to(dtype)
+    win = torch.randint(0, V, (N,), generator=g, device=dev)
+    wide[torch.arange(N, device=dev), col0 + win] += float(rng.choice([1.0, 6.0, 12.0]))
+    view = wide[:, col0:col0 + V]
+    blank, cap = int(rng.integers(0, V)), int(rng.choice([1, 50, 200, 600]))
+    kw = {}
+    if rng.random() < 0.4:
+        kw["ctas"] = int(rng.choice([1, 8, 37, 148]))
+    if rng.random() < 0.4:
+        kw["warps"] = int(rng.choice([1, 2, 5, 8, 12, 16]))
+    if rng.random() < 0.4:
+        kw["split"] = int(rng.choice([2, 4, 8, 16, 32]))
+    if rng.random() < 0.4 and dtype == torch.bfloat16:
+        kw["fma_exp"] = int(rng.choice([-1, 1, 2]))
+    try:
+        a = ssd.ssd_ctc_draft(view, off, blank, cap, V=V, opts=H.opts(**kw) if kw else None)
+    except ssd.SsdError as e:
+        assert e.code == ssd.ERR_ARG and "split" in kw       # a lane would walk too many chunks
+        return
+    b = ssd.ssd_ctc_draft(view, off, blank, cap, V=V, opts=H.opts(kernel=1))
+    torch.cuda.synchronize()
+    for k in ("frame_argmax", "draft_len", "draft_full_len", "utt_status"):
+        assert torch.equal(a[k], b[k]), k
+    assert not (H.status_u32(a["utt_status"]) != 0).any()
+    he, hp = a["frame_entropy"].double(), b["frame_entropy"].double()
+    assert float((he - hp).abs().max()) <= H.FLOAT_TOL
+    le, lp = a["frame_lse"].double(), b["frame_lse"].double()
+    assert float((le - lp).abs().max()) <= H.FLOAT_TOL + 2.5e-7 * float(lp.abs().max())
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_verify_kernels_agree_under_random_options(cuda_device, seed):
+    """ssd_verify's bulk-copy kernel under random launch options (grid, warps, column spans, ring
+    shape, exponential split, where rows are finished) against the plain-load kernel, on new
+    workspaces that hold whatever the allocator left in them."""
+    rng = np.random.default_rng(9000 + seed)
+    V = int(rng.choice([1, 9, 257, 1000, 4099, 32000, 50257]))
+    dtype = torch.bfloat16 if rng.random() < 0.6 else torch.float32
+    B = int(rng.choice([1, 2, 7, 32, 100, 257, 1000]))
+    lens = rng.integers(0, int(rng.choice([1, 3, 10, 60])) + 1, size=B)
+    if lens.sum() == 0:
+        lens[0] = 2
+    while lens.sum() * V > 1e8:
+        lens = lens // 2
+    M = int(lens.sum())
+    if M == 0:
+        lens[0] = 1
+        M = 1
+    off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    dev = cuda_device
+    pad = int(rng.integers(0, 9))
+    col0 = int(rng.integers(0, pad + 1))
+    g = torch.Generator(device=dev)
+    g.manual_seed(seed)
+    shift, scale = float(rng.choice([0.0, 0.0, -150.0, 90.0])), float(rng.choice([0.3, 2.0, 8.0]))
+    wide = (torch.randn((M, V + pad), generator=g, device=dev) * scale + shift).to(dtype)
+    ids = torch.randint(0, V, (M,), generator=g, device=dev, dtype=torch.int32)
+    keep = torch.rand((M,), generator=g, device=dev) < float(rng.choice([0.5, 0.97, 1.0]))
+    rows = torch.arange(M, device=dev)[keep]
+    wide[rows, col0 + ids[rows].long()] += float(rng.choice([6.0, 12.0, 30.0]))
+    view = wide[:, col0:col0 + V]
+    offd = torch.from_numpy(off).to(dev)
+    skip = (torch.rand((B,), generator=g, device=dev) < 0.3).to(torch.uint8) if rng.random() < 0.5 else None
+    kw = {}
+    if rng.random() < 0.3:
+        kw["ctas"] = int(rng.choice([1, 8, 37, 148]))
+    if rng.random() < 0.3:
+        kw["warps"] = int(rng.choice([1, 3, 4, 8, 12, 16]))
+    if rng.random() < 0.3:
+        kw["split"] = int(rng.choice([1, 2, 3, 7]))
+    if rng.random() < 0.3:
+        kw["stage_bytes"], kw["stages"] = int(rng.choice([1024, 4096, 16384, 65536])), int(rng.choice([2, 3, 5, 9]))
+    if rng.random() < 0.2 and dtype == torch.bfloat16:
+        kw["fma_exp"] = int(rng.choice([-1, 1, 2, 3]))
+    if rng.random() < 0.3:
+        kw["finish"], kw["split"] = 2, 1
+    tau = float(rng.choice([0.1, 0.2, 0.5]))
+    try:
+        a = ssd.ssd_verify(view, offd, ids, tau, skip=skip, V=V, opts=H.opts(**kw) if kw else None)
+    except ssd.SsdError as e:
+        assert e.code == ssd.ERR_ARG and kw           # a ring that does not fit, finish = 2 on too many utterances
+        return
+    b = ssd.ssd_verify(view, offd, ids, tau, skip=skip, V=V, opts=H.opts(kernel=1))
+    torch.cuda.synchronize()
+    sk = skip.cpu().numpy().astype(bool) if skip is not None else np.zeros(B, bool)
+    rowmask = torch.from_numpy(np.repeat(~sk, lens)).to(dev)
+    la, lb = a["token_logp"].double(), b["token_logp"].double()
+    fin = torch.isfinite(lb) & rowmask
+    if bool(fin.any()):
+        assert float((la[fin] - lb[fin]).abs().max()) <= 5e-5
+    if not bool((((lb - np.log(tau)).abs() < H.MARGIN) & rowmask).any()):
+        for k in ("accepted_len", "all_accepted", "utt_status"):
+            assert torch.equal(a[k], b[k]), k
